@@ -1,0 +1,179 @@
+"""CPU checker ("oracle"): ctypes front end of ulsnn_oracle.c.
+
+TEST INFRASTRUCTURE ONLY.  The product package never imports this; only the
+tests, the smoke check and the bench's CPU-baseline leg do.  It shares no code
+with the CUDA path.  Everything is computed in float64 from the fp32 inputs,
+directly from the definitions of Sections 3.1 and 4.1 (see the C file's header
+for what pins it).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ulsnn_oracle.c")
+_LIB = os.path.join(_HERE, "libulsnn_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C checker with gcc (-O2, OpenMP, no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", _LIB, _SRC, "-lm"]
+        subprocess.check_call(cmd)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        lib.oracle_sgemm_entry.restype = ctypes.c_double
+        lib.oracle_num_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _f32(a):
+    a = np.asarray(a)
+    assert a.dtype == np.float32, a.dtype
+    return a
+
+
+def _ptr(a, ct):
+    return a.ctypes.data_as(ctypes.POINTER(ct)) if a is not None else None
+
+
+def _trans(t) -> int:
+    t = str(t).upper()
+    assert t in ("N", "T"), t
+    return 1 if t == "T" else 0
+
+
+def sgemm(transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C=None, ldc=0) -> np.ndarray:
+    """C_out = alpha*op(A)*op(B) + beta*C in float64, dense [M, N] (Section 3.1)."""
+    A = _f32(A); B = _f32(B)
+    out = np.empty((M, N), dtype=np.float64)
+    if beta != 0.0:
+        C = _f32(C)
+    _load().oracle_sgemm(
+        ctypes.c_int(_trans(transA)), ctypes.c_int(_trans(transB)),
+        ctypes.c_int64(M), ctypes.c_int64(N), ctypes.c_int64(K), ctypes.c_double(alpha),
+        _ptr(A, ctypes.c_float), ctypes.c_int64(lda), _ptr(B, ctypes.c_float), ctypes.c_int64(ldb),
+        ctypes.c_double(beta), _ptr(C if beta != 0.0 else None, ctypes.c_float), ctypes.c_int64(ldc),
+        _ptr(out, ctypes.c_double))
+    return out
+
+
+def sgemm_entry(transA, transB, K, alpha, A, lda, B, ldb, beta, C, ldc, i, j) -> float:
+    A = _f32(A); B = _f32(B)
+    return float(_load().oracle_sgemm_entry(
+        ctypes.c_int(_trans(transA)), ctypes.c_int(_trans(transB)), ctypes.c_int64(K),
+        ctypes.c_double(alpha), _ptr(A, ctypes.c_float), ctypes.c_int64(lda),
+        _ptr(B, ctypes.c_float), ctypes.c_int64(ldb), ctypes.c_double(beta),
+        _ptr(_f32(C) if beta != 0.0 else None, ctypes.c_float), ctypes.c_int64(ldc),
+        ctypes.c_int64(i), ctypes.c_int64(j)))
+
+
+def _flatten(Ws, bs):
+    sizes = [int(Ws[0].shape[1])] + [int(w.shape[0]) for w in Ws]
+    for l, w in enumerate(Ws):
+        assert w.shape == (sizes[l + 1], sizes[l]) and bs[l].shape == (sizes[l + 1],)
+    Wflat = np.ascontiguousarray(np.concatenate([_f32(w).ravel() for w in Ws]))
+    bflat = np.ascontiguousarray(np.concatenate([_f32(b).ravel() for b in bs]))
+    return np.asarray(sizes, dtype=np.int32), Wflat, bflat
+
+
+def _unflatten(sizes, dW, db):
+    outW, outb, ow, ob = [], [], 0, 0
+    for l in range(len(sizes) - 1):
+        nw = int(sizes[l]) * int(sizes[l + 1])
+        outW.append(dW[ow:ow + nw].reshape(int(sizes[l + 1]), int(sizes[l]))); ow += nw
+        outb.append(db[ob:ob + int(sizes[l + 1])]); ob += int(sizes[l + 1])
+    return outW, outb
+
+
+def mlp_forward_loss(Ws, bs, X, labels) -> float:
+    """Summed cross-entropy of softmax(W_L h + b_L) over all patterns (no 1/n)."""
+    sizes, Wflat, bflat = _flatten(Ws, bs)
+    X = np.ascontiguousarray(_f32(X)); labels = np.ascontiguousarray(labels, dtype=np.int32)
+    loss = ctypes.c_double(0.0)
+    rc = _load().oracle_mlp_forward_loss(
+        ctypes.c_int(len(Ws)), _ptr(sizes, ctypes.c_int32), _ptr(Wflat, ctypes.c_float),
+        _ptr(bflat, ctypes.c_float), _ptr(X, ctypes.c_float), ctypes.c_int64(X.shape[1]),
+        _ptr(labels, ctypes.c_int32), ctypes.c_int64(X.shape[0]), ctypes.byref(loss))
+    assert rc == 0
+    return loss.value
+
+
+def mlp_gradient(Ws, bs, X, labels):
+    """(loss, [dW_l], [db_l]) summed over patterns, float64."""
+    sizes, Wflat, bflat = _flatten(Ws, bs)
+    X = np.ascontiguousarray(_f32(X)); labels = np.ascontiguousarray(labels, dtype=np.int32)
+    dW = np.zeros(Wflat.size, dtype=np.float64); db = np.zeros(bflat.size, dtype=np.float64)
+    loss = ctypes.c_double(0.0)
+    rc = _load().oracle_mlp_gradient(
+        ctypes.c_int(len(Ws)), _ptr(sizes, ctypes.c_int32), _ptr(Wflat, ctypes.c_float),
+        _ptr(bflat, ctypes.c_float), _ptr(X, ctypes.c_float), ctypes.c_int64(X.shape[1]),
+        _ptr(labels, ctypes.c_int32), ctypes.c_int64(X.shape[0]),
+        _ptr(dW, ctypes.c_double), _ptr(db, ctypes.c_double), ctypes.byref(loss))
+    assert rc == 0
+    gW, gb = _unflatten(sizes, dW, db)
+    return loss.value, gW, gb
+
+
+def mlp_sse_gradient(Ws, bs, X, T, want_grad=True):
+    """The paper's own head (tanh outputs, summed squared error, Eqs. 1 and 3)."""
+    sizes, Wflat, bflat = _flatten(Ws, bs)
+    X = np.ascontiguousarray(_f32(X)); T = np.ascontiguousarray(_f32(T))
+    dW = np.zeros(Wflat.size, dtype=np.float64); db = np.zeros(bflat.size, dtype=np.float64)
+    loss = ctypes.c_double(0.0)
+    rc = _load().oracle_mlp_sse_gradient(
+        ctypes.c_int(len(Ws)), _ptr(sizes, ctypes.c_int32), _ptr(Wflat, ctypes.c_float),
+        _ptr(bflat, ctypes.c_float), _ptr(X, ctypes.c_float), ctypes.c_int64(X.shape[1]),
+        _ptr(T, ctypes.c_float), ctypes.c_int64(T.shape[1]), ctypes.c_int64(X.shape[0]),
+        ctypes.c_int(1 if want_grad else 0),
+        _ptr(dW, ctypes.c_double), _ptr(db, ctypes.c_double), ctypes.byref(loss))
+    assert rc == 0
+    gW, gb = _unflatten(sizes, dW, db)
+    return loss.value, gW, gb
+
+
+def mlp_probe(Ws, bs, X, want_probs=True, want_hidden=True):
+    """Per-pattern softmax probabilities and last-hidden activations (float64)."""
+    sizes, Wflat, bflat = _flatten(Ws, bs)
+    X = np.ascontiguousarray(_f32(X))
+    n = X.shape[0]
+    probs = np.empty((n, int(sizes[-1])), dtype=np.float64) if want_probs else None
+    hid = np.empty((n, int(sizes[-2])), dtype=np.float64) if want_hidden else None
+    rc = _load().oracle_mlp_probe(
+        ctypes.c_int(len(Ws)), _ptr(sizes, ctypes.c_int32), _ptr(Wflat, ctypes.c_float),
+        _ptr(bflat, ctypes.c_float), _ptr(X, ctypes.c_float), ctypes.c_int64(X.shape[1]),
+        ctypes.c_int64(n), _ptr(probs, ctypes.c_double), _ptr(hid, ctypes.c_double))
+    assert rc == 0
+    return probs, hid
+
+
+def sgd_step(w, g, lr) -> np.ndarray:
+    """W - lr*grad evaluated in float64 and rounded once to fp32 (Section 4.2)."""
+    w = np.ascontiguousarray(_f32(w)); g = np.ascontiguousarray(_f32(g))
+    out = np.empty_like(w)
+    _load().oracle_sgd_step(ctypes.c_int64(w.size), _ptr(w, ctypes.c_float), _ptr(g, ctypes.c_float),
+                            ctypes.c_double(lr), _ptr(out, ctypes.c_float))
+    return out
+
+
+def rel_l2(x, ref) -> float:
+    """||x - ref||_2 / ||ref||_2 in float64 (absolute norm if ref is all zero)."""
+    x = np.asarray(x, dtype=np.float64).ravel(); ref = np.asarray(ref, dtype=np.float64).ravel()
+    d = np.linalg.norm(x - ref); r = np.linalg.norm(ref)
+    return float(d / r) if r > 0 else float(d)
