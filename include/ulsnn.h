@@ -1,0 +1,167 @@
+/*
+ * ulsnn — error-and-gradient evaluation of large fully connected networks by
+ * single-precision matrix products, on one NVIDIA B200 (sm_100a).
+ *
+ * The calls follow the problem statement of "Ultra-Large-Scale Neural-Network
+ * Training on a PIII Cluster": a Level-3-BLAS SGEMM (Section 3.1), "compute the
+ * error" and "compute the gradient" of a block of training patterns (Sections
+ * 4.2-4.3, 6.2) and the plain step W := W - alpha*grad (Section 4.2).
+ *
+ * Conventions that hold for every call
+ *  - Matrices are ROW-MAJOR fp32; a leading dimension (lda, ldx, ...) is the
+ *    distance in elements between consecutive rows (the "stride" of Section 3.4).
+ *  - Every data pointer is DEVICE memory owned by the caller, unless a comment
+ *    says "host".  Arrays of pointers (W, b, dW, db) are HOST arrays of device
+ *    pointers.  The library never frees or keeps a caller's buffer after the
+ *    work enqueued by a call has finished.
+ *  - Calls enqueue work on `stream` and return without synchronising.  They
+ *    never exit, throw or trap.  Argument errors are detected on the host
+ *    before anything is launched and reported through the return value.
+ *  - Results are bitwise reproducible from run to run: every reduction (split
+ *    K, column sums, loss) is done in an order fixed by the shapes only.
+ *  - Device-side waits are bounded; if one expires the kernel records it in a
+ *    status word and returns; ulsnn_last_device_status() reports it.
+ */
+#ifndef ULSNN_H
+#define ULSNN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int ulsnn_status_t;
+#define ULSNN_OK                        0
+#define ULSNN_ERR_INVALID_ARG          (-1)   /* bad trans, negative size, ld too small, null pointer, bad label range ... */
+#define ULSNN_ERR_UNSUPPORTED_ARCH     (-2)   /* current device is not compute capability 10.x */
+#define ULSNN_ERR_WORKSPACE_TOO_SMALL  (-3)
+#define ULSNN_ERR_CUDA                 (-4)   /* a CUDA runtime call failed (launch, attribute, allocation) */
+#define ULSNN_ERR_DEVICE_TIMEOUT       (-5)   /* a bounded device-side wait expired */
+#define ULSNN_ERR_TOO_LARGE            (-6)   /* a size exceeds a stated fixed maximum */
+
+/* How products of fp32 numbers are formed.  Accumulation is fp32 in all modes. */
+typedef enum {
+    ULSNN_MATH_3XTF32    = 0,  /* tensor cores, each operand split hi+lo in TF32, three products: fp32-level accuracy */
+    ULSNN_MATH_TF32      = 1,  /* tensor cores, operands truncated to TF32 (10-bit mantissa): fast mode */
+    ULSNN_MATH_FP32_SIMT = 2   /* FFMA on the CUDA cores: exact fp32 products, the comparison kernel */
+} ulsnn_math_t;
+
+/* A CUDA stream (cudaStream_t / CUstream); 0 is the legacy default stream. */
+typedef struct CUstream_st* ulsnn_stream_t;
+
+const char* ulsnn_status_string(ulsnn_status_t status);
+/* Packed version: major*10000 + minor*100 + patch. */
+int ulsnn_version(void);
+
+/* ------------------------------------------------------------------------------------------------
+ * SGEMM (Section 3.1: "C <- alpha*A*B + beta*C", 2MNK flops, Level-3 BLAS interface).
+ *
+ *   C = alpha * op(A) * op(B) + beta * C,   op(X) = X ('N'/'n') or X^T ('T'/'t')
+ *   op(A) is M x K, op(B) is K x N, C is M x N; row-major, so A is stored M x K with lda >= K when
+ *   transA == 'N' and K x M with lda >= M when transA == 'T' (likewise B with ldb >= N or >= K); ldc >= N.
+ *   beta == 0: C is overwritten and never read (it may hold NaN).  alpha == 0: A and B are not read.
+ *   M, N or K == 0 are valid (K == 0 gives C = beta*C).  A, B, C must not overlap.
+ *
+ * ulsnn_sgemm uses ULSNN_MATH_3XTF32.  For shapes with few output tiles and a long K it splits K and
+ * needs scratch memory: it takes it from a per-device buffer that the library allocates with cudaMalloc
+ * on first need and grows on demand (so that first call may synchronise the device, and must not happen
+ * inside a stream capture).  ulsnn_sgemm_ex never allocates: the caller passes the scratch
+ * (ulsnn_sgemm_workspace_bytes tells how much; workspace may be NULL when that is 0).  The workspace must be
+ * 256-byte aligned and may be reused by the next call on the same stream.
+ * Operands that the tensor-core path cannot address with TMA (a base pointer not 16-byte aligned, or a leading
+ * dimension that is not a multiple of 4) are computed by the FFMA kernel instead, which is at least as accurate.
+ * Errors: ULSNN_ERR_INVALID_ARG (nothing launched), ULSNN_ERR_WORKSPACE_TOO_SMALL, ULSNN_ERR_UNSUPPORTED_ARCH, ULSNN_ERR_CUDA.
+ */
+ulsnn_status_t ulsnn_sgemm(char transA, char transB, int64_t M, int64_t N, int64_t K, float alpha,
+                           const float* A, int64_t lda, const float* B, int64_t ldb,
+                           float beta, float* C, int64_t ldc, ulsnn_stream_t stream);
+ulsnn_status_t ulsnn_sgemm_ex(char transA, char transB, int64_t M, int64_t N, int64_t K, float alpha,
+                              const float* A, int64_t lda, const float* B, int64_t ldb,
+                              float beta, float* C, int64_t ldc, ulsnn_math_t math,
+                              void* workspace, size_t workspace_bytes, ulsnn_stream_t stream);
+ulsnn_status_t ulsnn_sgemm_workspace_bytes(char transA, char transB, int64_t M, int64_t N, int64_t K,
+                                           ulsnn_math_t math, size_t* bytes /* host, out */);
+
+/* ------------------------------------------------------------------------------------------------
+ * Network evaluation (Section 4.1, Eq. 2 for the tanh hidden layers; Section 4.2 for the matrix form
+ * H = tanh(X W^T), H_D = (1 - H*H)*(Y_D W), grad = H_D^T X, Y_D^T H; Section 4.3 for additivity over
+ * patterns).  The output layer is softmax with cross-entropy on integer labels, and every layer has a
+ * bias; with all biases zero the hidden layers are exactly Eq. 2.
+ *
+ * sizes[0..n_layers]: sizes[0] inputs, sizes[n_layers] classes, n_layers >= 1 weight matrices (<= 16).
+ * W[l] is [sizes[l+1] x sizes[l]] row-major dense (w_jk: j = unit of layer l+1, k = unit of layer l);
+ * b[l] is [sizes[l+1]].  max_patterns bounds n_patterns of every later call on the handle.
+ */
+typedef struct {
+    int32_t        n_layers;
+    const int32_t* sizes;         /* host, n_layers + 1 entries, each in [1, 2^20] */
+    ulsnn_math_t   math;
+    int64_t        max_patterns;  /* >= 1 */
+} ulsnn_mlp_desc_t;
+
+typedef struct ulsnn_mlp ulsnn_mlp_t;   /* opaque host object; owns no device memory */
+
+/* Device scratch the handle needs (activations, logits, deltas, split-K partials, row statistics). */
+ulsnn_status_t ulsnn_mlp_workspace_bytes(const ulsnn_mlp_desc_t* desc, size_t* bytes /* host, out */);
+/* workspace: device memory, 256-byte aligned, at least the size above; owned by the caller and borrowed by the
+ * handle until ulsnn_mlp_destroy.  Its contents are scratch between calls.  Calls on one handle must be
+ * stream-ordered with respect to each other (they share the workspace). */
+ulsnn_status_t ulsnn_mlp_create(ulsnn_mlp_t** handle /* host, out */, const ulsnn_mlp_desc_t* desc,
+                                void* workspace, size_t workspace_bytes);
+void           ulsnn_mlp_destroy(ulsnn_mlp_t* handle);
+
+/*
+ * "Compute the error": loss = sum_p [ logsumexp_j z_pj - z_{p,label_p} ], z = W_L h + b_L, SUMMED over the
+ * n_patterns patterns (no 1/n, as Eq. 3).  X is [n_patterns x sizes[0]] with ldx >= sizes[0]; labels are int32
+ * in [0, sizes[L]) (not checked on the host: an out-of-range label contributes as if no class matched).
+ * loss_out: device pointer to ONE double, written on the stream.  n_patterns == 0 writes 0.
+ * Costs 2*n_p*sum_l sizes[l]*sizes[l+1] flops (Section 6.2).
+ */
+ulsnn_status_t ulsnn_mlp_forward_loss(ulsnn_mlp_t* handle, const float* const* W, const float* const* b,
+                                      const float* X, int64_t ldx, const int32_t* labels, int64_t n_patterns,
+                                      double* loss_out, ulsnn_stream_t stream);
+/*
+ * "Compute the gradient": the loss above and its derivative with respect to every W[l] and b[l], summed over
+ * the patterns: dW[l] is [sizes[l+1] x sizes[l]] dense, db[l] is [sizes[l+1]].
+ * accumulate == 0: dW, db and *loss_out are overwritten.  accumulate != 0: the results of this block of patterns
+ * are ADDED to what dW, db and *loss_out hold (Section 4.3: error and gradient are additive over disjoint
+ * subsets of the training set); a caller sweeping a large training set chunk by chunk in a fixed order gets a
+ * bitwise reproducible total.  n_patterns == 0 with accumulate == 0 writes zeros.
+ */
+ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* handle, const float* const* W, const float* const* b,
+                                  const float* X, int64_t ldx, const int32_t* labels, int64_t n_patterns,
+                                  int accumulate, float* const* dW, float* const* db, double* loss_out,
+                                  ulsnn_stream_t stream);
+/* Section 4.2: W := W - lr * dW, b := b - lr * db, in place, one fused multiply-add per element. */
+ulsnn_status_t ulsnn_sgd_step(ulsnn_mlp_t* handle, float* const* W, float* const* b,
+                              const float* const* dW, const float* const* db, float lr, ulsnn_stream_t stream);
+/* Synchronises `stream`, then returns ULSNN_OK, ULSNN_ERR_DEVICE_TIMEOUT if a kernel of this handle gave up a
+ * bounded wait since the last call of this function (the word is cleared), or ULSNN_ERR_CUDA. */
+ulsnn_status_t ulsnn_last_device_status(ulsnn_mlp_t* handle, ulsnn_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Seeded synthetic data, generated in place on the device (no counterpart in the paper, whose data set is
+ * not available; used by the benchmarks to fill multi-gigabyte pattern matrices without a host copy).
+ * Element i of the tensor gets hash(seed, tensor_id, offset + i) mapped to
+ *   mode 0: uniform [0,1) on a 2^-24 grid;  mode 1: uniform [-1,1) on a 2^-23 grid.
+ * Labels: (hash >> 11) mod n_classes as int32.  The hash is a two-round splitmix64 finaliser of
+ * seed*0x9E3779B97F4A7C15 + tensor_id*0xD1B54A32D192ED03 + index + 1.
+ */
+ulsnn_status_t ulsnn_fill_uniform(float* dst, int64_t n, uint64_t seed, uint64_t tensor_id, uint64_t offset,
+                                  int mode, ulsnn_stream_t stream);
+ulsnn_status_t ulsnn_fill_labels(int32_t* dst, int64_t n, uint64_t seed, uint64_t tensor_id, uint64_t offset,
+                                 int32_t n_classes, ulsnn_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Instrumentation (no counterpart in the paper): number of kernel launches the library has enqueued since it
+ * was loaded, by kind.  counts (host, out): [0] FFMA GEMM kernels, [1] tcgen05 GEMM kernels, [2] reduction and
+ * other small kernels, [3] fill kernels.
+ */
+void ulsnn_launch_counts(int64_t counts[4]);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ULSNN_H */

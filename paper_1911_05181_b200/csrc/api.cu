@@ -1,0 +1,483 @@
+// C-ABI of the library: argument validation, workspace layout, and the stream-ordered sequence of
+// kernel launches that makes up one error / gradient evaluation (Section 4.2).
+#include "common.cuh"
+#include <atomic>
+#include <mutex>
+#include <new>
+#include <vector>
+
+namespace ulsnn {
+
+static std::atomic<int64_t> g_counts[4];
+void count_launch(int kind) { g_counts[kind & 3].fetch_add(1, std::memory_order_relaxed); }
+
+namespace {
+
+constexpr int MAX_LAYERS = 16;
+constexpr int64_t SLICE_CAP = 4096;     // longest run of patterns summed in one fp32 accumulator
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+bool parse_trans(char c, bool* t) {
+    if (c == 'N' || c == 'n') { *t = false; return true; }
+    if (c == 'T' || c == 't') { *t = true; return true; }
+    return false;
+}
+
+ulsnn_status_t check_arch() {
+    static std::mutex mu;
+    static int cached[64];          // 0 unknown, 1 ok, 2 unsupported
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ULSNN_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return ULSNN_ERR_UNSUPPORTED_ARCH;
+    std::lock_guard<std::mutex> lk(mu);
+    if (cached[dev] == 0) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ULSNN_ERR_CUDA;
+        cached[dev] = (major == 10) ? 1 : 2;
+    }
+    return cached[dev] == 1 ? ULSNN_OK : ULSNN_ERR_UNSUPPORTED_ARCH;
+}
+
+// Which engine computes a product asked for in `math`.
+bool use_tc(const GemmDesc& d, ulsnn_math_t math) {
+    return math != ULSNN_MATH_FP32_SIMT && tc_gemm_supported(d);
+}
+
+ulsnn_status_t run_gemm(const GemmDesc& d, ulsnn_math_t math, cudaStream_t stream) {
+    if (use_tc(d, math)) return tc_gemm_launch(d, math == ULSNN_MATH_3XTF32, stream);
+    return simt_gemm_launch(d, stream);
+}
+
+struct SplitPlan { int splits; int64_t k_per_split; };
+
+// Fixed by the shapes only.  Slices are at most SLICE_CAP long once K is large (bounds the fp32 rounding of a
+// long sum), and short-and-wide products get enough slices to fill the GPU.
+SplitPlan plan_splits(int64_t tiles, int64_t K) {
+    int64_t s_acc = (K > 2 * SLICE_CAP) ? (K + SLICE_CAP - 1) / SLICE_CAP : 1;
+    int64_t s_fill = 1;
+    if (tiles < 148 && K >= 1024) {
+        s_fill = (296 + tiles - 1) / tiles;
+        if (s_fill > K / 512) s_fill = K / 512;
+        if (s_fill < 1) s_fill = 1;
+    }
+    int64_t s = s_acc > s_fill ? s_acc : s_fill;
+    int64_t kps = round_up((K + s - 1) / s, 32);
+    if (kps < 32) kps = 32;
+    s = (K + kps - 1) / kps;
+    if (s < 1) s = 1;
+    return SplitPlan{(int)s, kps};
+}
+
+int64_t tiles_of(const GemmDesc& d, bool tc) {
+    const int64_t bm = tc ? tc_tile_m() : simt_tile_m();
+    const int64_t bn = tc ? tc_tile_n(d) : simt_tile_n();
+    return ((d.M + bm - 1) / bm) * ((d.N + bn - 1) / bn);
+}
+
+// ------------------------------------------------------------------------------------------- SGEMM
+
+struct SgemmArgs {
+    bool ta, tb; int64_t M, N, K; float alpha, beta;
+    const float* A; int64_t lda; const float* B; int64_t ldb; float* C; int64_t ldc;
+};
+
+ulsnn_status_t validate_sgemm(char transA, char transB, int64_t M, int64_t N, int64_t K,
+                              int64_t lda, int64_t ldb, int64_t ldc, bool* ta, bool* tb) {
+    if (!parse_trans(transA, ta) || !parse_trans(transB, tb)) return ULSNN_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || K < 0) return ULSNN_ERR_INVALID_ARG;
+    const int64_t a_cols = *ta ? M : K, b_cols = *tb ? K : N;
+    if (lda < (a_cols > 1 ? a_cols : 1) || ldb < (b_cols > 1 ? b_cols : 1) || ldc < (N > 1 ? N : 1)) return ULSNN_ERR_INVALID_ARG;
+    return ULSNN_OK;
+}
+
+GemmDesc sgemm_desc(const SgemmArgs& a) {
+    GemmDesc d{};
+    d.M = a.M; d.N = a.N; d.K = a.K;
+    d.A = a.A; d.a_sm = a.ta ? 1 : a.lda; d.a_sk = a.ta ? a.lda : 1;
+    d.B = a.B; d.b_sk = a.tb ? 1 : a.ldb; d.b_sn = a.tb ? a.ldb : 1;
+    d.C = a.C; d.ldc = a.ldc; d.alpha = a.alpha; d.beta = a.beta;
+    d.epi = EPI_SGEMM; d.splits = 1; d.k_per_split = a.K;
+    return d;
+}
+
+size_t sgemm_ws_for(const GemmDesc& d, bool tc) {
+    const SplitPlan p = plan_splits(tiles_of(d, tc), d.K);
+    if (p.splits <= 1) return 0;
+    return align256((size_t)p.splits * (size_t)d.M * (size_t)round_up(d.N, 4) * sizeof(float));
+}
+
+ulsnn_status_t sgemm_impl(const SgemmArgs& a, ulsnn_math_t math, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    if (a.M == 0 || a.N == 0) return ULSNN_OK;
+    if (!a.C) return ULSNN_ERR_INVALID_ARG;
+    if (a.K == 0 || a.alpha == 0.f) {
+        if (a.beta == 1.f) return ULSNN_OK;
+        return launch_scale_rows(a.C, a.M, a.N, a.ldc, a.beta, stream);
+    }
+    if (!a.A || !a.B) return ULSNN_ERR_INVALID_ARG;
+    GemmDesc d = sgemm_desc(a);
+    const bool tc = use_tc(d, math);
+    const SplitPlan p = plan_splits(tiles_of(d, tc), d.K);
+    if (p.splits <= 1) return run_gemm(d, math, stream);
+    const int64_t ldp = round_up(d.N, 4);
+    const size_t need = (size_t)p.splits * (size_t)d.M * (size_t)ldp * sizeof(float);
+    if (!ws || ws_bytes < need) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
+    if (((uintptr_t)ws & 255) != 0) return ULSNN_ERR_INVALID_ARG;
+    d.epi = EPI_PARTIAL; d.splits = p.splits; d.k_per_split = p.k_per_split;
+    d.partials = (float*)ws; d.ldp = ldp;
+    ulsnn_status_t st = run_gemm(d, math, stream);
+    if (st != ULSNN_OK) return st;
+    return launch_splitk_reduce(d.partials, p.splits, d.M, d.N, ldp, a.alpha, a.beta, a.C, a.ldc, nullptr, stream);
+}
+
+// grow-only scratch of ulsnn_sgemm, one per device
+struct DevScratch { void* p = nullptr; size_t bytes = 0; };
+DevScratch g_scratch[64];
+std::mutex g_scratch_mu;
+
+}  // namespace
+}  // namespace ulsnn
+
+using namespace ulsnn;
+
+// ----------------------------------------------------------------------------------------------- misc
+
+extern "C" const char* ulsnn_status_string(ulsnn_status_t s) {
+    switch (s) {
+        case ULSNN_OK: return "ok";
+        case ULSNN_ERR_INVALID_ARG: return "invalid argument";
+        case ULSNN_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x (B200)";
+        case ULSNN_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case ULSNN_ERR_CUDA: return "CUDA runtime error";
+        case ULSNN_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case ULSNN_ERR_TOO_LARGE: return "size exceeds a fixed maximum";
+    }
+    return "unknown status";
+}
+
+extern "C" int ulsnn_version(void) { return 100; }
+
+extern "C" void ulsnn_launch_counts(int64_t counts[4]) {
+    for (int i = 0; i < 4; ++i) counts[i] = g_counts[i].load(std::memory_order_relaxed);
+}
+
+// ----------------------------------------------------------------------------------------------- SGEMM
+
+extern "C" ulsnn_status_t ulsnn_sgemm_workspace_bytes(char transA, char transB, int64_t M, int64_t N, int64_t K,
+                                                      ulsnn_math_t math, size_t* bytes) {
+    bool ta, tb;
+    if (!bytes || !parse_trans(transA, &ta) || !parse_trans(transB, &tb) || M < 0 || N < 0 || K < 0) return ULSNN_ERR_INVALID_ARG;
+    if ((int)math < 0 || (int)math > 2) return ULSNN_ERR_INVALID_ARG;
+    *bytes = 0;
+    if (M == 0 || N == 0 || K == 0) return ULSNN_OK;
+    SgemmArgs a{ta, tb, M, N, K, 1.f, 0.f, nullptr, ta ? M : K, nullptr, tb ? K : N, nullptr, N};
+    a.lda = round_up(a.lda, 4); a.ldb = round_up(a.ldb, 4);       // an addressable stand-in for the tile-width query
+    GemmDesc d = sgemm_desc(a);
+    size_t w = sgemm_ws_for(d, false);
+    if (math != ULSNN_MATH_FP32_SIMT) { const size_t w2 = sgemm_ws_for(d, true); if (w2 > w) w = w2; }
+    *bytes = w;
+    return ULSNN_OK;
+}
+
+extern "C" ulsnn_status_t ulsnn_sgemm_ex(char transA, char transB, int64_t M, int64_t N, int64_t K, float alpha,
+                                         const float* A, int64_t lda, const float* B, int64_t ldb,
+                                         float beta, float* C, int64_t ldc, ulsnn_math_t math,
+                                         void* workspace, size_t workspace_bytes, ulsnn_stream_t stream) {
+    SgemmArgs a{false, false, M, N, K, alpha, beta, A, lda, B, ldb, C, ldc};
+    ulsnn_status_t st = validate_sgemm(transA, transB, M, N, K, lda, ldb, ldc, &a.ta, &a.tb);
+    if (st != ULSNN_OK) return st;
+    if ((int)math < 0 || (int)math > 2) return ULSNN_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return ULSNN_OK;
+    if ((st = check_arch()) != ULSNN_OK) return st;
+    return sgemm_impl(a, math, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+extern "C" ulsnn_status_t ulsnn_sgemm(char transA, char transB, int64_t M, int64_t N, int64_t K, float alpha,
+                                      const float* A, int64_t lda, const float* B, int64_t ldb,
+                                      float beta, float* C, int64_t ldc, ulsnn_stream_t stream) {
+    SgemmArgs a{false, false, M, N, K, alpha, beta, A, lda, B, ldb, C, ldc};
+    ulsnn_status_t st = validate_sgemm(transA, transB, M, N, K, lda, ldb, ldc, &a.ta, &a.tb);
+    if (st != ULSNN_OK) return st;
+    if (M == 0 || N == 0) return ULSNN_OK;
+    if ((st = check_arch()) != ULSNN_OK) return st;
+    void* ws = nullptr; size_t have = 0;
+    if (K > 0 && alpha != 0.f && A && B && C) {
+        GemmDesc d = sgemm_desc(a);
+        const size_t need = sgemm_ws_for(d, use_tc(d, ULSNN_MATH_3XTF32));
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ULSNN_ERR_CUDA;
+        std::lock_guard<std::mutex> lk(g_scratch_mu);
+        DevScratch& sc = g_scratch[dev];
+        if (need > sc.bytes) {
+            // cudaFree waits for all work on the device, so nothing still reads the old buffer
+            if (sc.p) cudaFree(sc.p);
+            sc.p = nullptr; sc.bytes = 0;
+            if (cudaMalloc(&sc.p, need) != cudaSuccess) { sc.p = nullptr; return ULSNN_ERR_CUDA; }
+            sc.bytes = need;
+        }
+        ws = sc.p; have = sc.bytes;
+    }
+    return sgemm_impl(a, ULSNN_MATH_3XTF32, ws, have, (cudaStream_t)stream);
+}
+
+// ----------------------------------------------------------------------------------------------- network
+
+struct ulsnn_mlp {
+    int L;
+    int32_t sizes[MAX_LAYERS + 1];
+    ulsnn_math_t math;
+    int64_t max_patterns;
+    // strides of the library-owned matrices
+    int64_t ldh[MAX_LAYERS + 1];    // H_l (output of weight l-1, l = 1..L-1): sizes[l] + a ones column, padded to 4
+    int64_t ldd[MAX_LAYERS + 1];    // delta_l, l = 1..L-1
+    int64_t ldz;                    // logits
+    int64_t stats_ld;
+    // workspace carve-up
+    float* H[MAX_LAYERS + 1];
+    float* D[MAX_LAYERS + 1];
+    float* Z;
+    float2* stats;
+    float* lse;
+    float* zlabel;
+    double* loss_parts;
+    float* colsum_parts;
+    float* partials;
+    size_t partials_bytes;
+    size_t total_bytes;
+};
+
+namespace {
+
+// Upper bound, over every batch length n <= B, of the split-K scratch for dW_w: M = sizes[w+1], N = sizes[w]
+// (+1 ones column when w >= 1).  plan_splits never returns more than max(ceil(n/SLICE_CAP), fill slices), and
+// both terms grow with n.
+size_t wgrad_partial_bound(const int32_t* sizes, int w, int64_t B) {
+    GemmDesc d{};
+    d.M = sizes[w + 1]; d.N = sizes[w] + (w >= 1 ? 1 : 0); d.K = B;
+    d.a_sm = 1; d.a_sk = 4; d.b_sk = 4; d.b_sn = 1;
+    const int64_t ldp = round_up(d.N, 4);
+    int64_t smax = (B + SLICE_CAP - 1) / SLICE_CAP;
+    for (int tc = 0; tc < 2; ++tc) {
+        const int64_t tiles = tiles_of(d, tc != 0);
+        if (tiles < 148 && B >= 1024) {
+            int64_t f = (296 + tiles - 1) / tiles;
+            if (f > B / 512) f = B / 512;
+            if (f > smax) smax = f;
+        }
+    }
+    if (smax < 1) smax = 1;
+    return (size_t)smax * (size_t)d.M * (size_t)ldp * sizeof(float);
+}
+
+ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
+    const int L = h->L; const int64_t B = h->max_patterns;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* p = base ? base + off : nullptr; off += align256(bytes); return p; };
+    for (int l = 1; l < L; ++l) {
+        h->ldh[l] = round_up((int64_t)h->sizes[l] + 1, 4);
+        h->ldd[l] = round_up((int64_t)h->sizes[l], 4);
+        h->H[l] = (float*)take((size_t)B * h->ldh[l] * sizeof(float));
+        h->D[l] = (float*)take((size_t)B * h->ldd[l] * sizeof(float));
+    }
+    h->ldz = round_up((int64_t)h->sizes[L], 4);
+    h->Z = (float*)take((size_t)B * h->ldz * sizeof(float));
+    h->stats_ld = ((int64_t)h->sizes[L] + 63) / 64;          // enough for any column-tile width >= 64
+    h->stats = (float2*)take((size_t)B * h->stats_ld * sizeof(float2));
+    h->lse = (float*)take((size_t)B * sizeof(float));
+    h->zlabel = (float*)take((size_t)B * sizeof(float));
+    h->loss_parts = (double*)take((size_t)(rowstats_blocks(B) + 1) * sizeof(double));
+    size_t cs = 0;
+    if (L >= 2) cs = (size_t)((B + 127) / 128) * (size_t)h->sizes[1] * sizeof(float);
+    else cs = (size_t)delta_colsum_tiles(B) * (size_t)h->sizes[1] * sizeof(float);
+    h->colsum_parts = (float*)take(cs);
+    size_t pb = 0;
+    for (int w = 0; w < L; ++w) { const size_t b = wgrad_partial_bound(h->sizes, w, B); if (b > pb) pb = b; }
+    h->partials_bytes = align256(pb);
+    h->partials = (float*)take(pb);
+    h->total_bytes = off;
+    return ULSNN_OK;
+}
+
+ulsnn_status_t check_desc(const ulsnn_mlp_desc_t* d) {
+    if (!d || !d->sizes || d->n_layers < 1 || d->n_layers > MAX_LAYERS || d->max_patterns < 1) return ULSNN_ERR_INVALID_ARG;
+    if ((int)d->math < 0 || (int)d->math > 2) return ULSNN_ERR_INVALID_ARG;
+    for (int l = 0; l <= d->n_layers; ++l) if (d->sizes[l] < 1 || d->sizes[l] > (1 << 20)) return ULSNN_ERR_INVALID_ARG;
+    if (d->max_patterns > ((int64_t)1 << 31) - 256) return ULSNN_ERR_TOO_LARGE;
+    return ULSNN_OK;
+}
+
+void fill_handle(ulsnn_mlp* h, const ulsnn_mlp_desc_t* d) {
+    *h = ulsnn_mlp{};
+    h->L = d->n_layers; h->math = d->math; h->max_patterns = d->max_patterns;
+    for (int l = 0; l <= h->L; ++l) h->sizes[l] = d->sizes[l];
+}
+
+// The forward products: hidden layers with bias + tanh fused, then the logits with their row statistics.
+ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
+                       const int32_t* labels, int64_t n, bool keep_logits, int accumulate, double* loss_out,
+                       cudaStream_t stream) {
+    const int L = h->L;
+    const float* in = X; int64_t ld_in = ldx;
+    for (int l = 1; l < L; ++l) {
+        GemmDesc d{};
+        d.M = n; d.N = h->sizes[l]; d.K = h->sizes[l - 1];
+        d.A = in; d.a_sm = ld_in; d.a_sk = 1;
+        d.B = W[l - 1]; d.b_sk = 1; d.b_sn = d.K;
+        d.C = h->H[l]; d.ldc = h->ldh[l]; d.alpha = 1.f; d.beta = 0.f;
+        d.epi = EPI_BIAS_TANH; d.bias = b[l - 1]; d.ones_cols = (int)(h->ldh[l] - d.N);
+        d.splits = 1; d.k_per_split = d.K;
+        ulsnn_status_t st = run_gemm(d, h->math, stream);
+        if (st != ULSNN_OK) return st;
+        in = h->H[l]; ld_in = h->ldh[l];
+    }
+    GemmDesc d{};
+    d.M = n; d.N = h->sizes[L]; d.K = h->sizes[L - 1];
+    d.A = in; d.a_sm = ld_in; d.a_sk = 1;
+    d.B = W[L - 1]; d.b_sk = 1; d.b_sn = d.K;
+    d.C = keep_logits ? h->Z : nullptr; d.ldc = h->ldz; d.alpha = 1.f; d.beta = 0.f;
+    d.epi = EPI_LOGITS; d.bias = b[L - 1]; d.labels = labels;
+    d.stats = h->stats; d.stats_ld = h->stats_ld; d.zlabel = h->zlabel;
+    d.splits = 1; d.k_per_split = d.K;
+    const bool tc = use_tc(d, h->math);
+    const int64_t bn = tc ? tc_tile_n(d) : simt_tile_n();
+    const int tiles = (int)((d.N + bn - 1) / bn);
+    if (tiles > h->stats_ld) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
+    ulsnn_status_t st = run_gemm(d, h->math, stream);
+    if (st != ULSNN_OK) return st;
+    return launch_rowstats(h->stats, h->stats_ld, tiles, h->zlabel, n, h->lse, h->loss_parts, accumulate, loss_out, stream);
+}
+
+ulsnn_status_t check_call(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
+                          const int32_t* labels, int64_t n, double* loss_out) {
+    if (!h || !W || !b || !loss_out || n < 0 || n > h->max_patterns) return ULSNN_ERR_INVALID_ARG;
+    if (n > 0 && (!X || !labels || ldx < h->sizes[0])) return ULSNN_ERR_INVALID_ARG;
+    for (int l = 0; l < h->L; ++l) if (!W[l] || !b[l]) return ULSNN_ERR_INVALID_ARG;
+    return ULSNN_OK;
+}
+
+}  // namespace
+
+extern "C" ulsnn_status_t ulsnn_mlp_workspace_bytes(const ulsnn_mlp_desc_t* desc, size_t* bytes) {
+    ulsnn_status_t st = check_desc(desc);
+    if (st != ULSNN_OK || !bytes) return st != ULSNN_OK ? st : ULSNN_ERR_INVALID_ARG;
+    ulsnn_mlp tmp; fill_handle(&tmp, desc);
+    layout(&tmp, nullptr);
+    *bytes = tmp.total_bytes;
+    return ULSNN_OK;
+}
+
+extern "C" ulsnn_status_t ulsnn_mlp_create(ulsnn_mlp_t** handle, const ulsnn_mlp_desc_t* desc, void* workspace, size_t workspace_bytes) {
+    if (!handle) return ULSNN_ERR_INVALID_ARG;
+    *handle = nullptr;
+    ulsnn_status_t st = check_desc(desc);
+    if (st != ULSNN_OK) return st;
+    if (!workspace || ((uintptr_t)workspace & 255) != 0) return ULSNN_ERR_INVALID_ARG;
+    ulsnn_mlp* h = new (std::nothrow) ulsnn_mlp;
+    if (!h) return ULSNN_ERR_CUDA;
+    fill_handle(h, desc);
+    layout(h, (char*)workspace);
+    if (h->total_bytes > workspace_bytes) { delete h; return ULSNN_ERR_WORKSPACE_TOO_SMALL; }
+    *handle = h;
+    return ULSNN_OK;
+}
+
+extern "C" void ulsnn_mlp_destroy(ulsnn_mlp_t* handle) { delete handle; }
+
+extern "C" ulsnn_status_t ulsnn_mlp_forward_loss(ulsnn_mlp_t* h, const float* const* W, const float* const* b,
+                                                 const float* X, int64_t ldx, const int32_t* labels, int64_t n,
+                                                 double* loss_out, ulsnn_stream_t stream_) {
+    cudaStream_t stream = (cudaStream_t)stream_;
+    ulsnn_status_t st = check_call(h, W, b, X, ldx, labels, n, loss_out);
+    if (st != ULSNN_OK) return st;
+    if ((st = check_arch()) != ULSNN_OK) return st;
+    if (n == 0) return launch_zero_f64(loss_out, 1, stream);
+    return forward(h, W, b, X, ldx, labels, n, false, 0, loss_out, stream);
+}
+
+extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const* W, const float* const* b,
+                                             const float* X, int64_t ldx, const int32_t* labels, int64_t n,
+                                             int accumulate, float* const* dW, float* const* db, double* loss_out,
+                                             ulsnn_stream_t stream_) {
+    cudaStream_t stream = (cudaStream_t)stream_;
+    ulsnn_status_t st = check_call(h, W, b, X, ldx, labels, n, loss_out);
+    if (st != ULSNN_OK) return st;
+    if (!dW || !db) return ULSNN_ERR_INVALID_ARG;
+    const int L = h->L;
+    for (int l = 0; l < L; ++l) if (!dW[l] || !db[l]) return ULSNN_ERR_INVALID_ARG;
+    if ((st = check_arch()) != ULSNN_OK) return st;
+    if (n == 0) {
+        if (accumulate) return ULSNN_OK;
+        for (int l = 0; l < L; ++l) {
+            if ((st = launch_zero(dW[l], (int64_t)h->sizes[l] * h->sizes[l + 1], stream)) != ULSNN_OK) return st;
+            if ((st = launch_zero(db[l], h->sizes[l + 1], stream)) != ULSNN_OK) return st;
+        }
+        return launch_zero_f64(loss_out, 1, stream);
+    }
+    if ((st = forward(h, W, b, X, ldx, labels, n, true, accumulate, loss_out, stream)) != ULSNN_OK) return st;
+
+    // Deltas of the hidden layers, top down: delta_l = (1 - H_l*H_l) * (delta_{l+1} W_{l+1})   (H_D of Section 4.2).
+    // delta_L is never stored: the kernels form softmax(z) - onehot from the logits as they load them.
+    for (int l = L - 1; l >= 1; --l) {
+        GemmDesc d{};
+        d.M = n; d.N = h->sizes[l]; d.K = h->sizes[l + 1];
+        if (l + 1 == L) { d.A = h->Z; d.a_sm = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 1; }
+        else            { d.A = h->D[l + 1]; d.a_sm = h->ldd[l + 1]; }
+        d.a_sk = 1;
+        d.B = W[l]; d.b_sk = d.N; d.b_sn = 1;
+        d.C = h->D[l]; d.ldc = h->ldd[l]; d.alpha = 1.f; d.beta = 0.f;
+        d.epi = EPI_TANHP; d.Hm = h->H[l]; d.ldh = h->ldh[l];
+        d.colsum_part = (l == 1) ? h->colsum_parts : nullptr;
+        d.splits = 1; d.k_per_split = d.K;
+        if ((st = run_gemm(d, h->math, stream)) != ULSNN_OK) return st;
+    }
+
+    // Weight gradients dW_w = delta_{w+1}^T * act_w: the sum over patterns is the K dimension (Section 4.2), cut into
+    // slices of a fixed length whose partial products are combined in slice order.
+    const float beta = accumulate ? 1.f : 0.f;
+    for (int w = L - 1; w >= 0; --w) {
+        GemmDesc d{};
+        d.M = h->sizes[w + 1]; d.N = h->sizes[w] + (w >= 1 ? 1 : 0); d.K = n;
+        if (w + 1 == L) { d.A = h->Z; d.a_sk = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 0; }
+        else            { d.A = h->D[w + 1]; d.a_sk = h->ldd[w + 1]; }
+        d.a_sm = 1;
+        if (w >= 1) { d.B = h->H[w]; d.b_sk = h->ldh[w]; } else { d.B = X; d.b_sk = ldx; }
+        d.b_sn = 1;
+        d.alpha = 1.f; d.beta = 0.f; d.epi = EPI_PARTIAL;
+        const SplitPlan p = plan_splits(tiles_of(d, use_tc(d, h->math)), d.K);
+        d.splits = p.splits; d.k_per_split = p.k_per_split;
+        d.ldp = round_up(d.N, 4); d.partials = h->partials;
+        if ((size_t)p.splits * (size_t)d.M * (size_t)d.ldp * sizeof(float) > h->partials_bytes) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
+        if ((st = run_gemm(d, h->math, stream)) != ULSNN_OK) return st;
+        if ((st = launch_splitk_reduce(d.partials, p.splits, d.M, h->sizes[w], d.ldp, 1.f, beta, dW[w], h->sizes[w],
+                                       w >= 1 ? db[w] : nullptr, stream)) != ULSNN_OK) return st;
+    }
+    // bias gradient of the first layer: column sums of delta_1 (both engines use 128-row tiles)
+    if (L >= 2) {
+        st = launch_colsum_reduce(h->colsum_parts, (n + 127) / 128, h->sizes[1], accumulate, db[0], stream);
+    } else {
+        st = launch_delta_colsum(h->Z, h->ldz, h->lse, labels, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);
+    }
+    return st;
+}
+
+extern "C" ulsnn_status_t ulsnn_sgd_step(ulsnn_mlp_t* h, float* const* W, float* const* b,
+                                         const float* const* dW, const float* const* db, float lr, ulsnn_stream_t stream) {
+    if (!h || !W || !b || !dW || !db) return ULSNN_ERR_INVALID_ARG;
+    for (int l = 0; l < h->L; ++l) if (!W[l] || !b[l] || !dW[l] || !db[l]) return ULSNN_ERR_INVALID_ARG;
+    ulsnn_status_t st = check_arch();
+    if (st != ULSNN_OK) return st;
+    for (int l = 0; l < h->L; ++l) {
+        if ((st = launch_sgd(W[l], dW[l], (int64_t)h->sizes[l] * h->sizes[l + 1], lr, (cudaStream_t)stream)) != ULSNN_OK) return st;
+        if ((st = launch_sgd(b[l], db[l], h->sizes[l + 1], lr, (cudaStream_t)stream)) != ULSNN_OK) return st;
+    }
+    return ULSNN_OK;
+}
+
+extern "C" ulsnn_status_t ulsnn_last_device_status(ulsnn_mlp_t* h, ulsnn_stream_t stream) {
+    (void)h;
+    int word = 0;
+    ulsnn_status_t st = device_status_fetch_and_clear((cudaStream_t)stream, &word);
+    if (st != ULSNN_OK) return st;
+    return word == DEV_OK ? ULSNN_OK : ULSNN_ERR_DEVICE_TIMEOUT;
+}

@@ -1,0 +1,89 @@
+// Shared declarations of the library's translation units (host + device).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/ulsnn.h"
+
+namespace ulsnn {
+
+// What a GEMM kernel does with its accumulator tile.
+enum Epilogue : int {
+    EPI_SGEMM     = 0,  // C = alpha*acc + beta*C                                   (Section 3.1)
+    EPI_BIAS_TANH = 1,  // C = tanh(acc + bias[col]); optionally C[:, N] = 1         (Eq. 2 / H = tanh(X W^T))
+    EPI_LOGITS    = 2,  // z = acc + bias[col]; per-(row, column-tile) softmax statistics, z at the label
+    EPI_TANHP     = 3,  // C = (1 - h*h) * acc, h = Hm[row][col]; per-row-tile column sums (H_D of Section 4.2)
+    EPI_PARTIAL   = 4   // split-K slice: raw accumulator into partials[slice]
+};
+
+// One product D = op(A) op(B) plus its fused epilogue; both engines (FFMA and tcgen05) take this.
+struct GemmDesc {
+    int64_t M, N, K;
+    const float* A; int64_t a_sm, a_sk;   // A(i,k) = A[i*a_sm + k*a_sk]  (one of the strides is 1)
+    const float* B; int64_t b_sk, b_sn;   // B(k,j) = B[k*b_sk + j*b_sn]
+    float* C; int64_t ldc;
+    float alpha, beta;
+    int epi;
+    // epilogue operands
+    const float* bias;        // [N]                 BIAS_TANH, LOGITS
+    int ones_cols;            // BIAS_TANH: write C[:, N] = 1 and C[:, N+1 .. N+ones_cols) = 0 (0: nothing)
+    const float* Hm; int64_t ldh;        // TANHP
+    float* colsum_part;       // TANHP: [row_tiles][N] partial column sums (may be null)
+    const int32_t* labels;    // LOGITS and the A transform: label of each pattern
+    float2* stats; int64_t stats_ld;     // LOGITS: stats[row*stats_ld + col_tile] = (max, sum exp(z - max))
+    float* zlabel;            // LOGITS: z[row][label[row]]
+    // A transform: the stored operand holds logits z; the product uses softmax(z) - onehot(label)
+    int a_transform;
+    const float* lse;         // [patterns] log-sum-exp of each pattern's logits
+    int a_pattern_is_m;       // 1: the M index of A is the pattern (K is the class); 0: K is the pattern
+    // split-K (EPI_PARTIAL): slice s covers k in [s*k_per_split, min(K, (s+1)*k_per_split))
+    int splits; int64_t k_per_split;
+    float* partials; int64_t ldp;        // partials[(s*M + i)*ldp + j]
+};
+
+// Device status word values (0 = fine).
+enum : int { DEV_OK = 0, DEV_TIMEOUT = 1 };
+
+// engines
+ulsnn_status_t simt_gemm_launch(const GemmDesc& d, cudaStream_t stream);
+int simt_tile_m();
+int simt_tile_n();
+// tcgen05 engine (tc_gemm.cu).  tc_gemm_supported: can TMA address these operands (16-byte aligned bases, leading
+// dimensions that are multiples of 4 floats)?  tc_tile_n: the column-tile width it will use for this product.
+bool tc_gemm_supported(const GemmDesc& d);
+int tc_tile_m();
+int tc_tile_n(const GemmDesc& d);
+ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stream);
+// device status word shared by all kernels of the library on the current device
+ulsnn_status_t device_status_fetch_and_clear(cudaStream_t stream, int* word);
+
+// reductions and small kernels (reduce.cu)
+// out[i*ldo + j] = alpha * sum_s parts[(s*M + i)*ldp + j] + beta*out   for j < N;   if bias_out: column N goes to
+// bias_out[i] (= sum_s parts[..][N], scaled the same way) -- the "ones column" that carries the bias gradient.
+ulsnn_status_t launch_splitk_reduce(const float* parts, int splits, int64_t M, int64_t N, int64_t ldp,
+                                    float alpha, float beta, float* out, int64_t ldo, float* bias_out,
+                                    cudaStream_t stream);
+// out[j] = sum_t parts[t*N + j] (+ out[j] if accumulate), t in fixed order
+ulsnn_status_t launch_colsum_reduce(const float* parts, int64_t tiles, int64_t N, int accumulate, float* out,
+                                    cudaStream_t stream);
+// lse[p] from the per-tile statistics; loss = sum_p (lse[p] - zlabel[p]) in a fixed order, in double
+ulsnn_status_t launch_rowstats(const float2* stats, int64_t stats_ld, int tiles, const float* zlabel, int64_t n,
+                               float* lse, double* block_partials, int accumulate, double* loss_out,
+                               cudaStream_t stream);
+int rowstats_blocks(int64_t n);
+// db[j] = sum_p softmax(z_p)_j - [label_p == j]   (only for networks without a hidden layer)
+ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* lse, const int32_t* labels,
+                                   int64_t n, int64_t n_classes, float* parts, int accumulate, float* out,
+                                   cudaStream_t stream);
+int delta_colsum_tiles(int64_t n);
+ulsnn_status_t launch_sgd(float* w, const float* g, int64_t n, float lr, cudaStream_t stream);
+ulsnn_status_t launch_zero(float* p, int64_t n, cudaStream_t stream);
+ulsnn_status_t launch_zero_f64(double* p, int64_t n, cudaStream_t stream);
+ulsnn_status_t launch_scale_rows(float* C, int64_t M, int64_t N, int64_t ldc, float beta, cudaStream_t stream);
+
+// launch accounting: kind 0 FFMA GEMM, 1 tcgen05 GEMM, 2 reductions/small kernels, 3 fills
+void count_launch(int kind);
+
+static inline ulsnn_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? ULSNN_OK : ULSNN_ERR_CUDA; }
+
+}  // namespace ulsnn

@@ -1,0 +1,241 @@
+// Fixed-order reductions and the small memory-bound kernels around the GEMMs.
+//
+// Every sum here is taken in an order that depends on the shapes only (never on arrival order), in
+// double where the number of terms is large, so repeated runs are bitwise identical (Section 4.3:
+// error and gradient are additive over patterns; this is the on-device form of that sum).
+#include "common.cuh"
+#include <math.h>
+
+namespace ulsnn {
+
+namespace {
+
+// out = alpha * sum_s parts[s] + beta*out, one thread per output element, slices in index order, sum in double.
+__global__ void splitk_reduce_kernel(const float* __restrict__ parts, int splits, int64_t M, int64_t N, int64_t ldp,
+                                     float alpha, float beta, float* __restrict__ out, int64_t ldo,
+                                     float* __restrict__ bias_out) {
+    const int64_t ncols = N + (bias_out ? 1 : 0);
+    const int64_t total = M * ncols;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = e / ncols, j = e - i * ncols;
+        double s = 0.0;
+        for (int sidx = 0; sidx < splits; ++sidx) s += (double)parts[((int64_t)sidx * M + i) * ldp + j];
+        float* dst = (j < N) ? out + i * ldo + j : bias_out + i;
+        double v = (double)alpha * s;
+        if (beta != 0.f) v += (double)beta * (double)*dst;
+        *dst = (float)v;
+    }
+}
+
+__global__ void colsum_reduce_kernel(const float* __restrict__ parts, int64_t tiles, int64_t N, int accumulate,
+                                     float* __restrict__ out) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= N) return;
+    double s = 0.0;
+    for (int64_t t = 0; t < tiles; ++t) s += (double)parts[t * N + j];
+    if (accumulate) s += (double)out[j];
+    out[j] = (float)s;
+}
+
+constexpr int RS_THREADS = 256;
+
+// One thread per pattern: combine the per-tile (max, sum-exp) pairs in tile order into the log-sum-exp,
+// then sum lse - z_label over the block in a fixed tree.
+__global__ void rowstats_kernel(const float2* __restrict__ stats, int64_t stats_ld, int tiles,
+                                const float* __restrict__ zlabel, int64_t n, float* __restrict__ lse,
+                                double* __restrict__ block_partials) {
+    __shared__ double red[RS_THREADS];
+    const int64_t p = (int64_t)blockIdx.x * RS_THREADS + threadIdx.x;
+    double term = 0.0;
+    if (p < n) {
+        float mx = -INFINITY;
+        for (int t = 0; t < tiles; ++t) mx = fmaxf(mx, stats[p * stats_ld + t].x);
+        double s = 0.0;
+        for (int t = 0; t < tiles; ++t) {
+            const float2 v = stats[p * stats_ld + t];
+            s += (double)v.y * exp((double)v.x - (double)mx);
+        }
+        const double l = (double)mx + log(s);
+        lse[p] = (float)l;
+        term = l - (double)zlabel[p];
+    }
+    red[threadIdx.x] = term;
+    __syncthreads();
+    for (int o = RS_THREADS / 2; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) block_partials[blockIdx.x] = red[0];
+}
+
+__global__ void loss_final_kernel(const double* __restrict__ block_partials, int nblocks, int accumulate,
+                                  double* __restrict__ loss_out) {
+    // a single thread: a few hundred additions in index order
+    double s = 0.0;
+    for (int i = 0; i < nblocks; ++i) s += block_partials[i];
+    *loss_out = accumulate ? *loss_out + s : s;
+}
+
+constexpr int DC_ROWS = 1024;   // patterns per partial row of the delta column sum
+
+__global__ void delta_colsum_kernel(const float* __restrict__ Z, int64_t ldz, const float* __restrict__ lse,
+                                    const int32_t* __restrict__ labels, int64_t n, int64_t n_classes,
+                                    float* __restrict__ parts) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n_classes) return;
+    const int64_t p0 = (int64_t)blockIdx.y * DC_ROWS, p1 = min(n, p0 + DC_ROWS);
+    float s = 0.f;
+    for (int64_t p = p0; p < p1; ++p) s += expf(Z[p * ldz + j] - lse[p]) - ((int64_t)labels[p] == j ? 1.f : 0.f);
+    parts[(int64_t)blockIdx.y * n_classes + j] = s;
+}
+
+__global__ void sgd_kernel(float* __restrict__ w, const float* __restrict__ g, int64_t n, float lr) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        w[i] = fmaf(-lr, g[i], w[i]);
+}
+
+template <typename T>
+__global__ void zero_kernel(T* __restrict__ p, int64_t n) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) p[i] = T(0);
+}
+
+__global__ void scale_rows_kernel(float* __restrict__ C, int64_t M, int64_t N, int64_t ldc, float beta) {
+    const int64_t total = M * N;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = e / N, j = e - i * N;
+        C[i * ldc + j] = (beta == 0.f) ? 0.f : beta * C[i * ldc + j];
+    }
+}
+
+__device__ __forceinline__ uint64_t mix64(uint64_t seed, uint64_t tensor_id, uint64_t index) {
+    uint64_t z = seed * 0x9E3779B97F4A7C15ull + tensor_id * 0xD1B54A32D192ED03ull + index + 1ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z = z ^ (z >> 31);
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z = z ^ (z >> 31);
+    return z;
+}
+
+__global__ void fill_uniform_kernel(float* __restrict__ dst, int64_t n, uint64_t seed, uint64_t tid, uint64_t offset, int mode) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint64_t h = mix64(seed, tid, offset + (uint64_t)i);
+        const float u = (float)(uint32_t)(h >> 40) * 5.9604644775390625e-8f;   // 2^-24, exact
+        dst[i] = mode ? 2.f * u - 1.f : u;
+    }
+}
+
+__global__ void fill_labels_kernel(int32_t* __restrict__ dst, int64_t n, uint64_t seed, uint64_t tid, uint64_t offset, uint32_t n_classes) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint64_t h = mix64(seed, tid, offset + (uint64_t)i);
+        dst[i] = (int32_t)((h >> 11) % (uint64_t)n_classes);
+    }
+}
+
+inline unsigned grid_for(int64_t n, int threads) {
+    int64_t b = (n + threads - 1) / threads;
+    if (b < 1) b = 1;
+    if (b > 148 * 16) b = 148 * 16;
+    return (unsigned)b;
+}
+
+}  // namespace
+
+ulsnn_status_t launch_splitk_reduce(const float* parts, int splits, int64_t M, int64_t N, int64_t ldp,
+                                    float alpha, float beta, float* out, int64_t ldo, float* bias_out,
+                                    cudaStream_t stream) {
+    if (M <= 0 || N <= 0) return ULSNN_OK;
+    splitk_reduce_kernel<<<grid_for(M * (N + 1), 256), 256, 0, stream>>>(parts, splits, M, N, ldp, alpha, beta, out, ldo, bias_out);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+ulsnn_status_t launch_colsum_reduce(const float* parts, int64_t tiles, int64_t N, int accumulate, float* out,
+                                    cudaStream_t stream) {
+    if (N <= 0) return ULSNN_OK;
+    colsum_reduce_kernel<<<(unsigned)((N + 127) / 128), 128, 0, stream>>>(parts, tiles, N, accumulate, out);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+int rowstats_blocks(int64_t n) { return (int)((n + RS_THREADS - 1) / RS_THREADS); }
+
+ulsnn_status_t launch_rowstats(const float2* stats, int64_t stats_ld, int tiles, const float* zlabel, int64_t n,
+                               float* lse, double* block_partials, int accumulate, double* loss_out,
+                               cudaStream_t stream) {
+    const int nb = rowstats_blocks(n);
+    if (nb > 0) {
+        rowstats_kernel<<<nb, RS_THREADS, 0, stream>>>(stats, stats_ld, tiles, zlabel, n, lse, block_partials);
+        ulsnn::count_launch(2);
+        if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
+    }
+    loss_final_kernel<<<1, 1, 0, stream>>>(block_partials, nb, accumulate, loss_out);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+int delta_colsum_tiles(int64_t n) { return (int)((n + DC_ROWS - 1) / DC_ROWS); }
+
+ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* lse, const int32_t* labels,
+                                   int64_t n, int64_t n_classes, float* parts, int accumulate, float* out,
+                                   cudaStream_t stream) {
+    const int tiles = delta_colsum_tiles(n);
+    if (tiles > 65535) return ULSNN_ERR_TOO_LARGE;
+    if (tiles > 0) {
+        dim3 grid((unsigned)((n_classes + 127) / 128), (unsigned)tiles);
+        delta_colsum_kernel<<<grid, 128, 0, stream>>>(Z, ldz, lse, labels, n, n_classes, parts);
+        ulsnn::count_launch(2);
+        if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
+    }
+    return launch_colsum_reduce(parts, tiles, n_classes, accumulate, out, stream);
+}
+
+ulsnn_status_t launch_sgd(float* w, const float* g, int64_t n, float lr, cudaStream_t stream) {
+    if (n <= 0) return ULSNN_OK;
+    sgd_kernel<<<grid_for(n, 256), 256, 0, stream>>>(w, g, n, lr);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+ulsnn_status_t launch_zero(float* p, int64_t n, cudaStream_t stream) {
+    if (n <= 0) return ULSNN_OK;
+    zero_kernel<float><<<grid_for(n, 256), 256, 0, stream>>>(p, n);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+ulsnn_status_t launch_zero_f64(double* p, int64_t n, cudaStream_t stream) {
+    if (n <= 0) return ULSNN_OK;
+    zero_kernel<double><<<grid_for(n, 256), 256, 0, stream>>>(p, n);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+ulsnn_status_t launch_scale_rows(float* C, int64_t M, int64_t N, int64_t ldc, float beta, cudaStream_t stream) {
+    if (M <= 0 || N <= 0) return ULSNN_OK;
+    scale_rows_kernel<<<grid_for(M * N, 256), 256, 0, stream>>>(C, M, N, ldc, beta);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace ulsnn
+
+extern "C" ulsnn_status_t ulsnn_fill_uniform(float* dst, int64_t n, uint64_t seed, uint64_t tensor_id, uint64_t offset,
+                                             int mode, ulsnn_stream_t stream) {
+    if (n < 0 || (n > 0 && !dst) || (mode != 0 && mode != 1)) return ULSNN_ERR_INVALID_ARG;
+    if (n == 0) return ULSNN_OK;
+    ulsnn::fill_uniform_kernel<<<ulsnn::grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(dst, n, seed, tensor_id, offset, mode);
+    ulsnn::count_launch(3);
+    return ulsnn::cuda_ok(cudaGetLastError());
+}
+
+extern "C" ulsnn_status_t ulsnn_fill_labels(int32_t* dst, int64_t n, uint64_t seed, uint64_t tensor_id, uint64_t offset,
+                                            int32_t n_classes, ulsnn_stream_t stream) {
+    if (n < 0 || (n > 0 && !dst) || n_classes < 1) return ULSNN_ERR_INVALID_ARG;
+    if (n == 0) return ULSNN_OK;
+    ulsnn::fill_labels_kernel<<<ulsnn::grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(dst, n, seed, tensor_id, offset, (uint32_t)n_classes);
+    ulsnn::count_launch(3);
+    return ulsnn::cuda_ok(cudaGetLastError());
+}
