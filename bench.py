@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the gradient evaluation (forward products, fused epilogues, delta products, weight-gradient
+products with their fixed-order reduction, then the plain step W -= lr*grad) on synthetic data shaped like
+the paper's 400-480-3203 character-recognition network.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--math 3xtf32|tf32|simt] [--workload config3|config1|config5]
+    python bench.py --impl reference ...      # times the CPU checker on the host cores instead
+
+One "step" = one error-and-gradient evaluation of one batch plus the parameter step.  Flops are counted with the
+paper's formula n_p*(4*n_i*n_h + 6*n_h*n_o) (Section 6.2), 2 per multiply-add, nothing else counted.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOADS = {
+    # name: (sizes, patterns per GPU, seed)
+    "config1": ([256, 128, 64], 4096, 0),
+    "config3": ([400, 480, 3203], 65536, 2),
+    "config5": ([1024, 4096, 4096, 3203], 131072, 4),
+}
+MATH = {"3xtf32": 0, "tf32": 1, "simt": 2}
+NOMINAL_TF32_OVER_BF16 = 0.5        # dense TF32 tensor rate is half the BF16 rate
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread:
+            self.thread.join(timeout=2)
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def cpu_baseline(sizes, seed, n_sample):
+    """The CPU checker, as it stands, on the first n_sample patterns of the workload."""
+    import oracle
+    import synth_inputs as si
+    from paper_1911_05181_b200 import flops
+    Ws, bs = si.mlp_params(seed, sizes)
+    X, y = si.mlp_batch(seed, sizes, n_sample)
+    t0 = time.perf_counter()
+    oracle.mlp_gradient(Ws, bs, X, y)
+    dt = time.perf_counter() - t0
+    return {"value": flops.gradient_flops(sizes, n_sample) / dt / 1e9, "unit": "GFLOP/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "sample": "first %d patterns of the batch, one gradient evaluation, %.1f s" % (n_sample, dt),
+            "patterns_per_s": n_sample / dt}
+
+
+def run_reference(args):
+    """--impl reference: the CPU checker on the host cores, same metric and config, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    import synth_inputs as si
+    from paper_1911_05181_b200 import flops
+    sizes, batch, seed = WORKLOADS[args.workload]
+    n_sample = min(batch, 2048 if args.workload != "config5" else 128)
+    Ws, bs = si.mlp_params(seed, sizes)
+    X, y = si.mlp_batch(seed, sizes, n_sample)
+    for _ in range(args.warmup):
+        oracle.mlp_gradient(Ws, bs, X, y)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        loss, dW, db = oracle.mlp_gradient(Ws, bs, X, y)
+        for w, g in zip(Ws + bs, dW + db):          # the parameter step, on a copy, so that every step sees the same weights
+            oracle.sgd_step(w.ravel(), g.astype("float32").ravel(), 1e-3 / n_sample)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = flops.gradient_flops(sizes, n_sample) / dt / 1e9
+    sample = "%d of %d patterns per step (work is additive over patterns)" % (n_sample, batch)
+    line = {
+        "impl": "reference", "metric": "gradient_eval_gflops", "value": val, "unit": "GFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s: %s MLP, %d patterns, seed %d" % (args.workload, "-".join(map(str, sizes)), batch, seed),
+                   "sample": sample},
+        "patterns_per_s": n_sample / dt,
+        "cpu_baseline": {"value": val, "unit": "GFLOP/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--math", default="3xtf32", choices=sorted(MATH))
+    ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    import synth_inputs as si
+    from paper_1911_05181_b200 import binding as ul, flops
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    ul.lib()                                       # raises if the CUDA library is not built: there is no other path
+
+    sizes, batch, seed = WORKLOADS[args.workload]
+    math_mode = MATH[args.math]
+    L = len(sizes) - 1
+    # Weak scaling (Section 4.3: patterns are partitioned, parameters replicated): every rank evaluates its own
+    # `batch` patterns, slice [rank*batch, (rank+1)*batch) of one seeded stream, and the gradients are summed.
+    Ws, bs = si.mlp_params(seed, sizes)
+    W = [torch.from_numpy(w).cuda() for w in Ws]
+    b = [torch.from_numpy(v).cuda() for v in bs]
+    W0 = [w.clone() for w in W]; b0 = [v.clone() for v in b]
+    dW = [torch.empty_like(w) for w in W]; db = [torch.empty_like(v) for v in b]
+    loss = torch.zeros(1, dtype=torch.float64, device="cuda")
+    X = torch.empty(batch, sizes[0], device="cuda"); y = torch.empty(batch, dtype=torch.int32, device="cuda")
+    ul.fill_uniform(X, X.numel(), seed, si.TID_X, rank * batch * sizes[0], 0)
+    ul.fill_labels(y, batch, seed, si.TID_LABELS, rank * batch, sizes[-1])
+    Xh = torch.empty(batch, sizes[0], pin_memory=True); yh = torch.empty(batch, dtype=torch.int32, pin_memory=True)
+    Xh.copy_(X); yh.copy_(y)
+    loss_h = torch.zeros(1, dtype=torch.float64, pin_memory=True)
+    net = ul.Mlp(sizes, math_mode, batch)
+    lr = 1e-3 / (batch * world)
+    stream = torch.cuda.current_stream()
+    flat = None
+    if world > 1:
+        flat = torch.empty(sum(t.numel() for t in dW + db), device="cuda")
+
+    def step(Xd, yd):
+        net.gradient(W, b, Xd, sizes[0], yd, batch, False, dW, db, loss)
+        if world > 1:
+            # the one exchange step of the method: sum of the per-rank gradients (Section 5), fp32, NCCL
+            torch.cat([t.reshape(-1) for t in dW + db], out=flat)
+            dist.all_reduce(flat)
+            off = 0
+            for t in dW + db:
+                t.copy_(flat[off:off + t.numel()].view_as(t)); off += t.numel()
+            dist.all_reduce(loss)
+        net.sgd_step(W, b, dW, db, lr)
+
+    def reset_params():
+        for w, w0 in zip(W + b, W0 + b0):
+            w.copy_(w0)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = float(t.item())
+        return ms / steps
+
+    # ---- device-resident throughput (inputs already in HBM; X 105 MB, logits 840 MB: far larger than the 126 MB L2)
+    for _ in range(max(args.warmup, 3)):
+        step(X, y)
+    reset_params()
+    net.enable_timing(True)
+    c0 = ul.launch_counts()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+    ms_step = timed(lambda: step(X, y), args.steps)
+    clocks = sampler.stop() if sampler else None
+    c1 = ul.launch_counts()
+    phases = net.phase_times()
+    net.enable_timing(False)
+    status = net.last_device_status()
+    launches = sum(c1[k] - c0[k] for k in c1)
+
+    # ---- end to end through the public call: inputs from pinned host memory every step, loss read back every step
+    reset_params()
+
+    def e2e_step():
+        X.copy_(Xh, non_blocking=True); y.copy_(yh, non_blocking=True)
+        step(X, y)
+        loss_h.copy_(loss, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    reset_params()
+    ms_e2e = timed(e2e_step, args.steps)
+
+    gflop_step = flops.gradient_flops(sizes, batch) * world / 1e9
+    value = gflop_step / (ms_step * 1e-3)
+    e2e_value = gflop_step / (ms_e2e * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant product (largest share of the step)
+    peaks = load_peaks()
+    dom = max(range(len(phases)), key=lambda i: phases[i][0]) if phases else None
+    roofline = None
+    if dom is not None:
+        ms_k, M, N, K = phases[dom]
+        logical = 2.0 * M * N * K
+        counts = ul.launch_counts()
+        on_tensor = args.math != "simt" and counts["tc_gemm"] > 0
+        if on_tensor:
+            mult = 3.0 if args.math == "3xtf32" else 1.0
+            peak = peaks["bf16_tflops_sustained"] * NOMINAL_TF32_OVER_BF16
+            achieved = mult * logical / (ms_k * 1e-3) / 1e12
+            roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                        "traffic": None, "kernel": "tc_gemm M=%d N=%d K=%d" % (M, N, K), "ms": ms_k,
+                        "flops_counted": "%gx 2MNK" % mult, "logical_tflops": logical / (ms_k * 1e-3) / 1e12,
+                        "peak_source": "%s cuBLAS bf16 sustained x 0.5 (nominal TF32:BF16)" % peaks["_source"]}
+        else:
+            sm_mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
+            peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12      # FFMA lanes x 2 flops x clock seen during the run
+            achieved = logical / (ms_k * 1e-3) / 1e12
+            roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                        "traffic": None, "kernel": "simt_gemm M=%d N=%d K=%d" % (M, N, K), "ms": ms_k,
+                        "peak_source": "148 SMs x 128 FFMA lanes x 2 x %.0f MHz (median SM clock of this run)" % sm_mhz}
+    gemm_ms = sum(p[0] for p in phases)
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        n_sample = {"config1": 4096, "config3": 16384, "config5": 1024}[args.workload]
+        cpu = cpu_baseline(sizes, seed, min(batch, n_sample))
+
+    line = {
+        "metric": "gradient_eval_gflops", "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "%s: %s MLP, %d patterns per GPU, seed %d" % (args.workload, "-".join(map(str, sizes)), batch, seed),
+                   "math": args.math, "global_batch": batch * world, "parallelism": "dp%d" % world,
+                   "l2": "inputs and intermediates (X 105 MB, logits 840 MB per step) exceed the 126 MB L2; no flush",
+                   "step": "gradient evaluation + W -= lr*grad, lr = 1e-3 / global_batch"},
+        "patterns_per_s": batch * world / (ms_step * 1e-3),
+        "pct_of_tf32_peak": None,
+        "e2e": {"value": e2e_value, "unit": "GFLOP/s", "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": Xh.numel() * 4 + yh.numel() * 4, "d2h_bytes_per_step": 8},
+        "gpu_launches": int(launches),
+        "launch_kinds": {k: int(c1[k] - c0[k]) for k in c1},
+        "roofline": roofline,
+        "phases_ms": [{"ms": round(p[0], 4), "M": p[1], "N": p[2], "K": p[3]} for p in phases],
+        "gemm_share_of_step": gemm_ms / ms_step if ms_step else None,
+        "cpu_baseline": cpu,
+        "clocks": clocks,
+        "device_status": status,
+        "peaks": {k: peaks.get(k) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "_source")},
+    }
+    tf32_peak = peaks["bf16_tflops_sustained"] * NOMINAL_TF32_OVER_BF16 * 1e3   # GFLOP/s
+    mult = 3.0 if args.math == "3xtf32" else 1.0
+    line["pct_of_tf32_peak"] = {"logical": 100.0 * value / world / tf32_peak,
+                                "tensor_pipe": 100.0 * mult * value / world / tf32_peak if args.math != "simt" else None,
+                                "peak_gflops": tf32_peak}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

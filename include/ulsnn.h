@@ -115,7 +115,8 @@ void           ulsnn_mlp_destroy(ulsnn_mlp_t* handle);
 /*
  * "Compute the error": loss = sum_p [ logsumexp_j z_pj - z_{p,label_p} ], z = W_L h + b_L, SUMMED over the
  * n_patterns patterns (no 1/n, as Eq. 3).  X is [n_patterns x sizes[0]] with ldx >= sizes[0]; labels are int32
- * in [0, sizes[L]) (not checked on the host: an out-of-range label contributes as if no class matched).
+ * in [0, sizes[L]) (not checked: with an out-of-range label the results are unspecified, but nothing is
+ * read or written out of bounds).
  * loss_out: device pointer to ONE double, written on the stream.  n_patterns == 0 writes 0.
  * Costs 2*n_p*sum_l sizes[l]*sizes[l+1] flops (Section 6.2).
  */
@@ -160,6 +161,18 @@ ulsnn_status_t ulsnn_fill_labels(int32_t* dst, int64_t n, uint64_t seed, uint64_
  * other small kernels, [3] fill kernels.
  */
 void ulsnn_launch_counts(int64_t counts[4]);
+/*
+ * Per-product device times of a handle (no counterpart in the paper).  With timing switched on, every GEMM launch of
+ * ulsnn_mlp_forward_loss / ulsnn_mlp_gradient is bracketed by CUDA events on the call's stream (the events are created
+ * when timing is first switched on).  Switching it on also resets the record.  ulsnn_mlp_phase_times waits for the
+ * recorded events and returns the device time of each product AVERAGED over the calls made since timing was switched
+ * on (at most the 64 most recent; all of them must have been calls of the same kind): n (host, in: capacity of the
+ * arrays, out: number of products), ms[i] the mean time of product i, mnk[3*i..3*i+2] its M, N, K.  Products come in
+ * launch order: the L forward products, the L-1 delta products (top layer first), the L weight-gradient products
+ * (top layer first).
+ */
+ulsnn_status_t ulsnn_mlp_enable_timing(ulsnn_mlp_t* handle, int on);
+ulsnn_status_t ulsnn_mlp_phase_times(ulsnn_mlp_t* handle, int* n, float* ms, int64_t* mnk);
 
 #ifdef __cplusplus
 }

@@ -29,7 +29,7 @@ EXPORTS = [
     "ulsnn_status_string", "ulsnn_version", "ulsnn_sgemm", "ulsnn_sgemm_ex", "ulsnn_sgemm_workspace_bytes",
     "ulsnn_mlp_workspace_bytes", "ulsnn_mlp_create", "ulsnn_mlp_destroy", "ulsnn_mlp_forward_loss",
     "ulsnn_mlp_gradient", "ulsnn_sgd_step", "ulsnn_last_device_status", "ulsnn_fill_uniform",
-    "ulsnn_fill_labels", "ulsnn_launch_counts",
+    "ulsnn_fill_labels", "ulsnn_launch_counts", "ulsnn_mlp_enable_timing", "ulsnn_mlp_phase_times",
 ]
 
 
@@ -76,6 +76,8 @@ def lib():
         l.ulsnn_fill_labels.argtypes = [vp, i64, u64, u64, u64, i32, vp]
         l.ulsnn_launch_counts.argtypes = [ctypes.POINTER(i64)]
         l.ulsnn_launch_counts.restype = None
+        l.ulsnn_mlp_enable_timing.argtypes = [vp, ctypes.c_int]
+        l.ulsnn_mlp_phase_times.argtypes = [vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(f32), ctypes.POINTER(i64)]
         _lib = l
     return _lib
 
@@ -211,6 +213,16 @@ class Mlp:
         if check:
             _check(st, "ulsnn_sgd_step")
         return st
+
+    def enable_timing(self, on=True):
+        _check(lib().ulsnn_mlp_enable_timing(self._h, 1 if on else 0), "ulsnn_mlp_enable_timing")
+
+    def phase_times(self):
+        """[(ms, M, N, K)] of the products of the most recent forward_loss / gradient call (timing must be on)."""
+        cap = 64
+        n = ctypes.c_int(cap); ms = (ctypes.c_float * cap)(); mnk = (ctypes.c_int64 * (3 * cap))()
+        _check(lib().ulsnn_mlp_phase_times(self._h, ctypes.byref(n), ms, mnk), "ulsnn_mlp_phase_times")
+        return [(ms[i], mnk[3 * i], mnk[3 * i + 1], mnk[3 * i + 2]) for i in range(n.value)]
 
     def last_device_status(self, stream=None) -> int:
         return lib().ulsnn_last_device_status(self._h, _stream(stream))

@@ -14,6 +14,7 @@ void count_launch(int kind) { g_counts[kind & 3].fetch_add(1, std::memory_order_
 namespace {
 
 constexpr int MAX_LAYERS = 16;
+constexpr int TIMING_SLOTS = 64;        // per-product timings are kept for this many most recent calls
 constexpr int64_t SLICE_CAP = 4096;     // longest run of patterns summed in one fp32 accumulator
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
@@ -245,6 +246,12 @@ struct ulsnn_mlp {
     float* partials;
     size_t partials_bytes;
     size_t total_bytes;
+    // optional per-product timing
+    bool timing;
+    int n_phases;                       // products launched so far by the call in flight
+    int64_t timed_calls;                // calls recorded since timing was switched on
+    std::vector<cudaEvent_t> ev;        // [TIMING_SLOTS][3*MAX_LAYERS][2], slot = call index modulo TIMING_SLOTS
+    int64_t phase_mnk[3 * (3 * MAX_LAYERS)];
 };
 
 namespace {
@@ -313,11 +320,26 @@ void fill_handle(ulsnn_mlp* h, const ulsnn_mlp_desc_t* d) {
     for (int l = 0; l <= h->L; ++l) h->sizes[l] = d->sizes[l];
 }
 
+// run_gemm bracketed by events when the handle's timing is on
+ulsnn_status_t timed_gemm(ulsnn_mlp* h, const GemmDesc& d, cudaStream_t stream) {
+    if (!h->timing || h->n_phases >= 3 * MAX_LAYERS) return run_gemm(d, h->math, stream);
+    const int i = h->n_phases++;
+    h->phase_mnk[3 * i] = d.M; h->phase_mnk[3 * i + 1] = d.N; h->phase_mnk[3 * i + 2] = d.K;
+    const size_t slot = (size_t)((h->timed_calls - 1) % TIMING_SLOTS);
+    cudaEvent_t* e = &h->ev[(slot * 3 * MAX_LAYERS + i) * 2];
+    if (cudaEventRecord(e[0], stream) != cudaSuccess) return ULSNN_ERR_CUDA;
+    ulsnn_status_t st = run_gemm(d, h->math, stream);
+    if (cudaEventRecord(e[1], stream) != cudaSuccess) return ULSNN_ERR_CUDA;
+    return st;
+}
+
 // The forward products: hidden layers with bias + tanh fused, then the logits with their row statistics.
 ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
                        const int32_t* labels, int64_t n, bool keep_logits, int accumulate, double* loss_out,
                        cudaStream_t stream) {
     const int L = h->L;
+    h->n_phases = 0;
+    if (h->timing) h->timed_calls++;
     const float* in = X; int64_t ld_in = ldx;
     for (int l = 1; l < L; ++l) {
         GemmDesc d{};
@@ -327,7 +349,7 @@ ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* 
         d.C = h->H[l]; d.ldc = h->ldh[l]; d.alpha = 1.f; d.beta = 0.f;
         d.epi = EPI_BIAS_TANH; d.bias = b[l - 1]; d.ones_cols = (int)(h->ldh[l] - d.N);
         d.splits = 1; d.k_per_split = d.K;
-        ulsnn_status_t st = run_gemm(d, h->math, stream);
+        ulsnn_status_t st = timed_gemm(h, d, stream);
         if (st != ULSNN_OK) return st;
         in = h->H[l]; ld_in = h->ldh[l];
     }
@@ -343,7 +365,7 @@ ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* 
     const int64_t bn = tc ? tc_tile_n(d) : simt_tile_n();
     const int tiles = (int)((d.N + bn - 1) / bn);
     if (tiles > h->stats_ld) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
-    ulsnn_status_t st = run_gemm(d, h->math, stream);
+    ulsnn_status_t st = timed_gemm(h, d, stream);
     if (st != ULSNN_OK) return st;
     return launch_rowstats(h->stats, h->stats_ld, tiles, h->zlabel, n, h->lse, h->loss_parts, accumulate, loss_out, stream);
 }
@@ -382,7 +404,50 @@ extern "C" ulsnn_status_t ulsnn_mlp_create(ulsnn_mlp_t** handle, const ulsnn_mlp
     return ULSNN_OK;
 }
 
-extern "C" void ulsnn_mlp_destroy(ulsnn_mlp_t* handle) { delete handle; }
+extern "C" void ulsnn_mlp_destroy(ulsnn_mlp_t* handle) {
+    if (!handle) return;
+    for (cudaEvent_t e : handle->ev) if (e) cudaEventDestroy(e);
+    delete handle;
+}
+
+extern "C" ulsnn_status_t ulsnn_mlp_enable_timing(ulsnn_mlp_t* h, int on) {
+    if (!h) return ULSNN_ERR_INVALID_ARG;
+    if (on && h->ev.empty()) {
+        h->ev.assign((size_t)TIMING_SLOTS * 3 * MAX_LAYERS * 2, nullptr);
+        const size_t used = (size_t)(3 * h->L - 1) * 2;
+        for (int slot = 0; slot < TIMING_SLOTS; ++slot)
+            for (size_t i = 0; i < used; ++i)
+                if (cudaEventCreate(&h->ev[(size_t)slot * 3 * MAX_LAYERS * 2 + i]) != cudaSuccess) return ULSNN_ERR_CUDA;
+    }
+    h->timing = on != 0;
+    h->n_phases = 0;
+    h->timed_calls = 0;
+    return ULSNN_OK;
+}
+
+extern "C" ulsnn_status_t ulsnn_mlp_phase_times(ulsnn_mlp_t* h, int* n, float* ms, int64_t* mnk) {
+    if (!h || !n || !ms || !mnk || *n < 0) return ULSNN_ERR_INVALID_ARG;
+    const int cap = *n;
+    *n = 0;
+    if (!h->timing || h->timed_calls == 0) return ULSNN_OK;
+    const int cnt = h->n_phases < cap ? h->n_phases : cap;
+    const int64_t calls = h->timed_calls < TIMING_SLOTS ? h->timed_calls : TIMING_SLOTS;
+    for (int i = 0; i < cnt; ++i) {
+        double sum = 0.0;
+        for (int64_t c = 0; c < calls; ++c) {
+            const size_t slot = (size_t)((h->timed_calls - 1 - c) % TIMING_SLOTS);
+            cudaEvent_t* e = &h->ev[(slot * 3 * MAX_LAYERS + i) * 2];
+            float t = 0.f;
+            if (cudaEventSynchronize(e[1]) != cudaSuccess) return ULSNN_ERR_CUDA;
+            if (cudaEventElapsedTime(&t, e[0], e[1]) != cudaSuccess) return ULSNN_ERR_CUDA;
+            sum += t;
+        }
+        ms[i] = (float)(sum / (double)calls);
+        for (int j = 0; j < 3; ++j) mnk[3 * i + j] = h->phase_mnk[3 * i + j];
+    }
+    *n = cnt;
+    return ULSNN_OK;
+}
 
 extern "C" ulsnn_status_t ulsnn_mlp_forward_loss(ulsnn_mlp_t* h, const float* const* W, const float* const* b,
                                                  const float* X, int64_t ldx, const int32_t* labels, int64_t n,
@@ -429,7 +494,7 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
         d.epi = EPI_TANHP; d.Hm = h->H[l]; d.ldh = h->ldh[l];
         d.colsum_part = (l == 1) ? h->colsum_parts : nullptr;
         d.splits = 1; d.k_per_split = d.K;
-        if ((st = run_gemm(d, h->math, stream)) != ULSNN_OK) return st;
+        if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
     }
 
     // Weight gradients dW_w = delta_{w+1}^T * act_w: the sum over patterns is the K dimension (Section 4.2), cut into
@@ -448,7 +513,7 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
         d.splits = p.splits; d.k_per_split = p.k_per_split;
         d.ldp = round_up(d.N, 4); d.partials = h->partials;
         if ((size_t)p.splits * (size_t)d.M * (size_t)d.ldp * sizeof(float) > h->partials_bytes) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
-        if ((st = run_gemm(d, h->math, stream)) != ULSNN_OK) return st;
+        if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
         if ((st = launch_splitk_reduce(d.partials, p.splits, d.M, h->sizes[w], d.ldp, 1.f, beta, dW[w], h->sizes[w],
                                        w >= 1 ? db[w] : nullptr, stream)) != ULSNN_OK) return st;
     }
