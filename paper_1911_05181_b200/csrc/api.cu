@@ -295,7 +295,7 @@ ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
     h->zlabel = (float*)take((size_t)B * sizeof(float));
     h->loss_parts = (double*)take((size_t)(rowstats_blocks(B) + 1) * sizeof(double));
     size_t cs = 0;
-    if (L >= 2) cs = (size_t)((B + 127) / 128) * (size_t)h->sizes[1] * sizeof(float);
+    if (L >= 2) cs = (size_t)((B + 127) / 128) * 4 * (size_t)h->sizes[1] * sizeof(float);
     else cs = (size_t)delta_colsum_tiles(B) * (size_t)h->sizes[1] * sizeof(float);
     h->colsum_parts = (float*)take(cs);
     size_t pb = 0;
@@ -481,6 +481,7 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
     }
     if ((st = forward(h, W, b, X, ldx, labels, n, true, accumulate, loss_out, stream)) != ULSNN_OK) return st;
 
+    int64_t colsum_rows = 0;
     // Deltas of the hidden layers, top down: delta_l = (1 - H_l*H_l) * (delta_{l+1} W_{l+1})   (H_D of Section 4.2).
     // delta_L is never stored: the kernels form softmax(z) - onehot from the logits as they load them.
     for (int l = L - 1; l >= 1; --l) {
@@ -494,6 +495,7 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
         d.epi = EPI_TANHP; d.Hm = h->H[l]; d.ldh = h->ldh[l];
         d.colsum_part = (l == 1) ? h->colsum_parts : nullptr;
         d.splits = 1; d.k_per_split = d.K;
+        if (l == 1) colsum_rows = ((n + 127) / 128) * (use_tc(d, h->math) ? tc_colsum_groups() : simt_colsum_groups());
         if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
     }
 
@@ -519,7 +521,7 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
     }
     // bias gradient of the first layer: column sums of delta_1 (both engines use 128-row tiles)
     if (L >= 2) {
-        st = launch_colsum_reduce(h->colsum_parts, (n + 127) / 128, h->sizes[1], accumulate, db[0], stream);
+        st = launch_colsum_reduce(h->colsum_parts, colsum_rows, h->sizes[1], accumulate, db[0], stream);
     } else {
         st = launch_delta_colsum(h->Z, h->ldz, h->lse, labels, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);
     }

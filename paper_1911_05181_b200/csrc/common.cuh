@@ -28,7 +28,7 @@ struct GemmDesc {
     const float* bias;        // [N]                 BIAS_TANH, LOGITS
     int ones_cols;            // BIAS_TANH: write C[:, N] = 1 and C[:, N+1 .. N+ones_cols) = 0 (0: nothing)
     const float* Hm; int64_t ldh;        // TANHP
-    float* colsum_part;       // TANHP: [row_tiles][N] partial column sums (may be null)
+    float* colsum_part;       // TANHP: [row_tiles * groups][N] partial column sums (may be null)
     const int32_t* labels;    // LOGITS and the A transform: label of each pattern
     float2* stats; int64_t stats_ld;     // LOGITS: stats[row*stats_ld + col_tile] = (max, sum exp(z - max))
     float* zlabel;            // LOGITS: z[row][label[row]]
@@ -53,6 +53,9 @@ int simt_tile_n();
 bool tc_gemm_supported(const GemmDesc& d);
 int tc_tile_m();
 int tc_tile_n(const GemmDesc& d);
+// EPI_TANHP writes this many partial column-sum rows per 128-row tile (row index = tile*groups + group)
+int tc_colsum_groups();
+int simt_colsum_groups();
 ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stream);
 // device status word shared by all kernels of the library on the current device
 ulsnn_status_t device_status_fetch_and_clear(cudaStream_t stream, int* word);

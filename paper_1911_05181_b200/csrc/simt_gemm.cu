@@ -221,6 +221,7 @@ ulsnn_status_t launch(const GemmDesc& d, cudaStream_t stream) {
 
 int simt_tile_m() { return BM; }
 int simt_tile_n() { return BN; }
+int simt_colsum_groups() { return 1; }
 
 ulsnn_status_t simt_gemm_launch(const GemmDesc& d, cudaStream_t stream) {
     if (d.M <= 0 || d.N <= 0) return ULSNN_OK;
