@@ -126,6 +126,8 @@ def run_reference(args):
     import synth_inputs as si
     from paper_1911_05181_b200 import flops
     sizes, batch, seed = WORKLOADS[args.workload]
+    if args.patterns > 0:
+        batch = args.patterns
     n_sample = min(batch, 2048 if args.workload != "config5" else 128)
     Ws, bs = si.mlp_params(seed, sizes)
     X, y = si.mlp_batch(seed, sizes, n_sample)
@@ -163,6 +165,8 @@ def main():
     ap.add_argument("--math", default="3xtf32", choices=sorted(MATH))
     ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--patterns", type=int, default=0,
+                    help="patterns per GPU instead of the workload's own count (for profiler captures of a smaller case)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -183,6 +187,8 @@ def main():
     ul.lib()                                       # raises if the CUDA library is not built: there is no other path
 
     sizes, batch, seed = WORKLOADS[args.workload]
+    if args.patterns > 0:
+        batch = args.patterns
     math_mode = MATH[args.math]
     L = len(sizes) - 1
     # Weak scaling (Section 4.3: patterns are partitioned, parameters replicated): every rank evaluates its own
