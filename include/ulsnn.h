@@ -84,6 +84,30 @@ ulsnn_status_t ulsnn_sgemm_ex(char transA, char transB, int64_t M, int64_t N, in
 ulsnn_status_t ulsnn_sgemm_workspace_bytes(char transA, char transB, int64_t M, int64_t N, int64_t K,
                                            ulsnn_math_t math, size_t* bytes /* host, out */);
 
+/*
+ * SGEMM for callers that cannot allocate device memory (the paper has no counterpart of this call).
+ *
+ * Some callers have no way to provide scratch: code that runs where cudaMalloc is off limits (inside a region
+ * whose memory budget is fixed up front, under a host framework that owns every allocation, in a callback that
+ * must not synchronise the device) cannot size and pass the workspace ulsnn_sgemm_ex wants, and cannot accept
+ * the allocate-on-first-need of ulsnn_sgemm.  ulsnn_sgemm_noalloc computes the same product as ulsnn_sgemm_ex with
+ * the same `math`, but takes its split-K scratch from a fixed array of ulsnn_sgemm_noalloc_max_scratch_bytes()
+ * (8 MiB) that is part of the library's image on every GPU that loads it.  It calls neither cudaMalloc nor
+ * cudaFree nor any allocating routine.
+ *  - A product whose split-K partials do not fit (ulsnn_sgemm_workspace_bytes(...) > the maximum) is rejected
+ *    with ULSNN_ERR_TOO_LARGE and nothing is launched.  Products that need no split never touch the array.
+ *  - The first call on each device that needs the array looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents (nothing has to start
+ *    at zero: every slice overwrites what the reduction reads).  Calls that could overlap on the GPU (different
+ *    streams without an ordering between them) race on it: keep them on one stream or order them yourself.
+ * Other arguments, conventions and errors are those of ulsnn_sgemm_ex.
+ */
+size_t         ulsnn_sgemm_noalloc_max_scratch_bytes(void);
+ulsnn_status_t ulsnn_sgemm_noalloc(char transA, char transB, int64_t M, int64_t N, int64_t K, float alpha,
+                                   const float* A, int64_t lda, const float* B, int64_t ldb,
+                                   float beta, float* C, int64_t ldc, ulsnn_math_t math, ulsnn_stream_t stream);
+
 /* ------------------------------------------------------------------------------------------------
  * Network evaluation (Section 4.1, Eq. 2 for the tanh hidden layers; Section 4.2 for the matrix form
  * H = tanh(X W^T), H_D = (1 - H*H)*(Y_D W), grad = H_D^T X, Y_D^T H; Section 4.3 for additivity over

@@ -30,6 +30,7 @@ EXPORTS = [
     "ulsnn_mlp_workspace_bytes", "ulsnn_mlp_create", "ulsnn_mlp_destroy", "ulsnn_mlp_forward_loss",
     "ulsnn_mlp_gradient", "ulsnn_sgd_step", "ulsnn_last_device_status", "ulsnn_fill_uniform",
     "ulsnn_fill_labels", "ulsnn_launch_counts", "ulsnn_mlp_enable_timing", "ulsnn_mlp_phase_times",
+    "ulsnn_sgemm_noalloc", "ulsnn_sgemm_noalloc_max_scratch_bytes",
 ]
 
 
@@ -61,6 +62,9 @@ def lib():
         l.ulsnn_version.restype = ctypes.c_int
         l.ulsnn_sgemm.argtypes = [ctypes.c_char, ctypes.c_char, i64, i64, i64, f32, vp, i64, vp, i64, f32, vp, i64, vp]
         l.ulsnn_sgemm_ex.argtypes = l.ulsnn_sgemm.argtypes[:-1] + [ctypes.c_int, vp, sz, vp]
+        l.ulsnn_sgemm_noalloc.argtypes = l.ulsnn_sgemm.argtypes[:-1] + [ctypes.c_int, vp]
+        l.ulsnn_sgemm_noalloc_max_scratch_bytes.restype = sz
+        l.ulsnn_sgemm_noalloc_max_scratch_bytes.argtypes = []
         l.ulsnn_sgemm_workspace_bytes.argtypes = [ctypes.c_char, ctypes.c_char, i64, i64, i64, ctypes.c_int,
                                                   ctypes.POINTER(sz)]
         l.ulsnn_mlp_workspace_bytes.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(sz)]
@@ -144,6 +148,20 @@ def sgemm_ex(transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, math=
                               beta, _ptr(C), ldc, math, _ptr(workspace), workspace_bytes, _stream(stream))
     if check:
         _check(st, "ulsnn_sgemm_ex")
+    return st
+
+
+def sgemm_noalloc_max_scratch_bytes() -> int:
+    return int(lib().ulsnn_sgemm_noalloc_max_scratch_bytes())
+
+
+def sgemm_noalloc(transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, math=MATH_3XTF32, stream=None,
+                  check=True):
+    """ulsnn_sgemm_noalloc: the product of sgemm_ex with the split-K scratch taken from the library's fixed array."""
+    st = lib().ulsnn_sgemm_noalloc(transA.encode(), transB.encode(), M, N, K, alpha, _ptr(A), lda, _ptr(B), ldb,
+                                   beta, _ptr(C), ldc, math, _stream(stream))
+    if check:
+        _check(st, "ulsnn_sgemm_noalloc")
     return st
 
 

@@ -222,6 +222,61 @@ extern "C" ulsnn_status_t ulsnn_sgemm(char transA, char transB, int64_t M, int64
     return sgemm_impl(a, ULSNN_MATH_3XTF32, ws, have, (cudaStream_t)stream);
 }
 
+// ----------------------------------------------------------------------------------------------- SGEMM without allocation
+
+// Split-K scratch of ulsnn_sgemm_noalloc.  It lives in the library's image: every device that loads the library
+// holds these bytes until the process exits, which is why the size is kept modest.
+#define ULSNN_NOALLOC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[ULSNN_NOALLOC_SCRATCH_BYTES];
+
+namespace ulsnn {
+namespace {
+// In host code `g_noalloc_scratch` is only a handle of the symbol; the address a kernel can use has to be asked for,
+// per device, with that device current.
+std::mutex g_noalloc_mu;
+void* g_noalloc_ptr[64];
+
+ulsnn_status_t noalloc_scratch(void** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ULSNN_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return ULSNN_ERR_CUDA;
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return ULSNN_OK;
+}
+}  // namespace
+}  // namespace ulsnn
+
+extern "C" size_t ulsnn_sgemm_noalloc_max_scratch_bytes(void) { return (size_t)ULSNN_NOALLOC_SCRATCH_BYTES; }
+
+extern "C" ulsnn_status_t ulsnn_sgemm_noalloc(char transA, char transB, int64_t M, int64_t N, int64_t K, float alpha,
+                                              const float* A, int64_t lda, const float* B, int64_t ldb,
+                                              float beta, float* C, int64_t ldc, ulsnn_math_t math,
+                                              ulsnn_stream_t stream) {
+    SgemmArgs a{false, false, M, N, K, alpha, beta, A, lda, B, ldb, C, ldc};
+    ulsnn_status_t st = validate_sgemm(transA, transB, M, N, K, lda, ldb, ldc, &a.ta, &a.tb);
+    if (st != ULSNN_OK) return st;
+    if ((int)math < 0 || (int)math > 2) return ULSNN_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return ULSNN_OK;
+    size_t need = 0;
+    if (K > 0 && alpha != 0.f && A && B && C) {
+        // the same slice plan as ulsnn_sgemm_ex makes for these operands, so the two give the same bits
+        GemmDesc d = sgemm_desc(a);
+        need = sgemm_ws_for(d, use_tc(d, math));
+    }
+    if (need > (size_t)ULSNN_NOALLOC_SCRATCH_BYTES) return ULSNN_ERR_TOO_LARGE;
+    if ((st = check_arch()) != ULSNN_OK) return st;
+    void* ws = nullptr;
+    if (need > 0 && (st = noalloc_scratch(&ws)) != ULSNN_OK) return st;
+    // Every slice writes all the entries of its partial product that the reduction reads, so the scratch needs
+    // no clearing although it still holds what the previous call left there.
+    return sgemm_impl(a, math, ws, need, (cudaStream_t)stream);
+}
+
 // ----------------------------------------------------------------------------------------------- network
 
 struct ulsnn_mlp {
