@@ -4,9 +4,14 @@
 // One persistent CTA per SM, 14 warps with fixed roles:
 //   warp 0      TMA producer      global -> 128B-swizzled shared-memory stages (cp.async.bulk.tensor, no multicast)
 //   warp 1      MMA issuer        one thread issues tcgen05.mma.kind::tf32 (128 x BN x 8 per instruction)
-//   warps 2-5   epilogue          tcgen05.ld of the 128 x BN fp32 accumulator (one row per thread), fused math, stores
+//   warps 2-5   epilogue          tcgen05.ld of the 128 x BN fp32 accumulator (one row per thread), fused math, then
+//                                 32x32 blocks staged in swizzled shared memory and written with TMA stores
+//                                 (whole 128-byte lines, edges clipped by the tensor map)
 //   warps 6-13  operand pass      only in 3xTF32 mode or when A is formed from logits: reads a landed stage,
-//                                 writes hi = tf32(x) in place and lo = tf32(x - hi) beside it
+//                                 rewrites it as hi = tf32_rn(x) and writes lo = tf32(x - hi) beside it.  (The
+//                                 tensor core ignores the low 13 mantissa bits of an fp32 word, so the landed tile
+//                                 could serve as hi = trunc(x) unchanged; the lo parts then all have the sign of x
+//                                 and the accumulator's truncation no longer averages out: measured 2.4x the error.)
 // TMEM holds two 256-column accumulator regions.  A tile's total lives in one of them, so its epilogue overlaps
 // the products of the next tile, which uses the other.  The tensor core adds into an fp32 accumulator with
 // truncation, a bias that grows with the number of instructions chained on one accumulator; in 3xTF32 mode the
@@ -22,6 +27,7 @@
 #include "common.cuh"
 #include <cuda.h>
 #include <math.h>
+#include <string.h>
 #include <mutex>
 
 namespace ulsnn {
@@ -41,13 +47,15 @@ constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 8;
 constexpr int A_TILE_BYTES = BM * BK * 4;                       // 16 KB
 constexpr int SMEM_BUDGET = 227 * 1024;
-constexpr int EPI_SCRATCH_BYTES = NUM_EPI_WARPS * 32 * 33 * 4;   // column-sum staging, one padded 32x32 tile per warp
+constexpr int EPI_STAGE_BYTES = 32 * 128;                        // one 32x32 fp32 block, 128B-swizzled
+constexpr int EPI_SCRATCH_BYTES = NUM_EPI_WARPS * 2 * EPI_STAGE_BYTES;   // two store-staging blocks per epilogue warp
 constexpr int CTRL_BYTES = 1024;                                // barriers, TMEM base, abort flag
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 3000000000ull; // ~1.5 s at 2 GHz
 
 struct TcParams {
     GemmDesc d;
-    int bn;                 // column-tile width (multiple of 16; multiple of 32 when B is MN-major)
+    int bn;                 // column-tile width, a multiple of 32 (the last tile of a row may use fewer columns)
+    int n_gran;             // granularity of the width the tensor core is given for that last tile: 16, or 32 when B is MN-major
     int tiles_m, tiles_n;
     int units;              // tiles_m * tiles_n * splits
     int stages;
@@ -56,6 +64,8 @@ struct TcParams {
     int three_x, a_mn, b_mn, split_pass;
     int chunk_blocks;       // k-blocks accumulated on one TMEM accumulator before it is added into the tile total
     int fast_math;          // TF32 mode: approximate exp
+    int round_hi;           // 3xTF32: the operand pass also rewrites the landed tile as hi = tf32_rn(x) (lo = x - hi)
+    int c_tma;              // the output (C or the split-K partials) is written with TMA stores
     int64_t n_patterns, n_classes;      // bounds of the logits operand when a_transform
     int* status;
 };
@@ -86,6 +96,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
 }
@@ -196,6 +213,12 @@ __device__ __forceinline__ void unit_coords(const TcParams& p, int u, int& mt, i
     sp = r / p.tiles_m;
 }
 
+// columns of column tile nt that the products cover: the whole tile, or what is left of the matrix rounded up
+__device__ __forceinline__ int tile_cols(const TcParams& p, int nt) {
+    const int left = (int)p.d.N - nt * p.bn;
+    return left >= p.bn ? p.bn : (left + p.n_gran - 1) / p.n_gran * p.n_gran;
+}
+
 __device__ __forceinline__ void unit_k_range(const TcParams& p, int sp, int64_t& kbeg, int& nkb, int& tail_steps) {
     kbeg = (p.d.epi == EPI_PARTIAL) ? (int64_t)sp * p.d.k_per_split : 0;
     int64_t kend = (p.d.epi == EPI_PARTIAL) ? kbeg + p.d.k_per_split : p.d.K;
@@ -206,15 +229,77 @@ __device__ __forceinline__ void unit_k_range(const TcParams& p, int sp, int64_t&
     tail_steps = (rem + UMMA_K - 1) / UMMA_K;
 }
 
+// Ring position: stage index and the parity of the pass over the ring.
+struct RingPos {
+    int stage; uint32_t phase;
+    __device__ __forceinline__ void advance(int stages) { if (++stage == stages) { stage = 0; phase ^= 1u; } }
+};
+
+// Sum over the 32 lanes of a warp of each of 32 per-lane values: lane l ends up with the total of v[l].
+// A butterfly of five exchange steps, so the order of the additions is fixed.
+__device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const bool up = lane & 16;
+        const float send = up ? v[j] : v[j + 16], keep = up ? v[j + 16] : v[j];
+        v[j] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const bool up = lane & 8;
+        const float send = up ? v[j] : v[j + 8], keep = up ? v[j + 8] : v[j];
+        v[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const bool up = lane & 4;
+        const float send = up ? v[j] : v[j + 4], keep = up ? v[j + 4] : v[j];
+        v[j] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const bool up = lane & 2;
+        const float send = up ? v[j] : v[j + 2], keep = up ? v[j + 2] : v[j];
+        v[j] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+    }
+    {
+        const bool up = lane & 1;
+        const float send = up ? v[0] : v[1], keep = up ? v[1] : v[0];
+        v[0] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+    }
+    return v[0];
+}
+
+// softmax(z) - onehot from a stored logit: e = exp(z - lse) - [cls == label], 0 outside the matrix
+__device__ __forceinline__ float delta_of(float z, float lse, int cls, int label, int n_classes, int fast) {
+    return (cls < n_classes) ? exp_mode(z - lse, fast) - (cls == label ? 1.f : 0.f) : 0.f;
+}
+
+__device__ __forceinline__ float lo_part(float x) {
+    return to_tf32(x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u));
+}
+// hi/lo parts of four values: with round_hi the hi part is rounded to nearest and has to be written back,
+// otherwise it is the truncation the tensor core applies to the stored word by itself
+__device__ __forceinline__ void split4(const float4 x, bool round_hi, float4& hi, float4& lo) {
+    if (round_hi) {
+        hi = make_float4(to_tf32(x.x), to_tf32(x.y), to_tf32(x.z), to_tf32(x.w));
+        lo = make_float4(to_tf32(x.x - hi.x), to_tf32(x.y - hi.y), to_tf32(x.z - hi.z), to_tf32(x.w - hi.w));
+    } else {
+        hi = x;
+        lo = make_float4(lo_part(x.x), lo_part(x.y), lo_part(x.z), lo_part(x.w));
+    }
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p) {
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_c, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128B swizzle pattern repeats every 8 rows of 128 bytes
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* stage_base = smem;
-    float* epi_scratch = (float*)(smem + (size_t)p.stages * p.stage_bytes);
-    Ctrl* ctrl = (Ctrl*)((uint8_t*)epi_scratch + EPI_SCRATCH_BYTES);
+    uint8_t* epi_scratch = smem + (size_t)p.stages * p.stage_bytes;
+    Ctrl* ctrl = (Ctrl*)(epi_scratch + EPI_SCRATCH_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const GemmDesc& d = p.d;
@@ -241,39 +326,43 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
 
-    // offsets inside a stage
+    // offsets inside a stage: the landed A and B tiles, then (3xTF32) their lo parts
     const int off_a_hi = 0, off_b_hi = A_TILE_BYTES;
     const int off_a_lo = A_TILE_BYTES + p.b_tile_bytes, off_b_lo = 2 * A_TILE_BYTES + p.b_tile_bytes;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t it = 0;
+            RingPos rp{0, 0};
             bool ok = true;
-            const uint32_t tx_bytes = (uint32_t)(A_TILE_BYTES + p.b_tile_bytes);
             for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
                 int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
                 int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
                 const int m0 = mt * BM, n0 = nt * p.bn;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % p.stages;
-                    const uint32_t ph = (it / p.stages) & 1;
-                    if (!wait_bar(&ctrl->empty[s], ph ^ 1, ctrl, p.status)) { ok = false; break; }
+                // a K-major B tile is one box of bn rows (rows past the matrix arrive as zeros); an MN-major one is a
+                // box per 32 columns, and only the boxes the products read are fetched
+                const int b_boxes = tile_cols(p, nt) >> 5;
+                const uint32_t tx_bytes = (uint32_t)(A_TILE_BYTES + (p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes));
+                int k0 = (int)kbeg;
+                for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
+                    const int s = rp.stage;
+                    if (!wait_bar(&ctrl->empty[s], rp.phase ^ 1, ctrl, p.status)) { ok = false; break; }
+                    rp.advance(p.stages);
                     const uint32_t bar = smem_u32(&ctrl->full[s]);
                     mbar_expect_tx(bar, tx_bytes);
                     const uint32_t sa = smem_u32(stage_base + (size_t)s * p.stage_bytes + off_a_hi);
-                    const uint32_t sb = smem_u32(stage_base + (size_t)s * p.stage_bytes + off_b_hi);
-                    const int k0 = (int)(kbeg + (int64_t)kb * BK);
+                    const uint32_t sb = sa + off_b_hi;
                     if (!p.a_mn) {
                         tma_load_2d(sa, &map_a, k0, m0, bar);                       // box {32 k, 128 rows}
                     } else {
+#pragma unroll
                         for (int g = 0; g < BM / 32; ++g)                           // boxes {32 m, 32 k}
                             tma_load_2d(sa + g * (BK * 128), &map_a, m0 + 32 * g, k0, bar);
                     }
                     if (!p.b_mn) {
                         tma_load_2d(sb, &map_b, k0, n0, bar);                       // box {32 k, bn rows}
                     } else {
-                        for (int g = 0; g < p.bn / 32; ++g)
+                        for (int g = 0; g < b_boxes; ++g)
                             tma_load_2d(sb + g * (BK * 128), &map_b, n0 + 32 * g, k0, bar);
                     }
                 }
@@ -282,8 +371,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
-                                   ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            const uint32_t idesc0 = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
+                                    ((uint32_t)(BM >> 4) << 24);
             // K-major (128B swizzle): 8-row groups 1024 B apart (SBO), K advance = 32 B inside the swizzled row.
             // MN-major (128B swizzle, 32-byte atoms): 32-element groups BK*128 B apart (LBO), 4-k groups 512 B apart
             // (SBO), K advance = 8 rows = 1024 B.
@@ -291,16 +380,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t a_sbo = p.a_mn ? 512 : 1024, b_sbo = p.b_mn ? 512 : 1024;
             const uint32_t a_lay = p.a_mn ? 1 : 2, b_lay = p.b_mn ? 1 : 2;
             const uint32_t a_kstep = p.a_mn ? 1024 : UMMA_K * 4, b_kstep = p.b_mn ? 1024 : UMMA_K * 4;
-            uint32_t it = 0, tile_i = 0;
+            // descriptors of the four tiles of stage 0; a stage or a k step only moves the 14-bit start address
+            const uint32_t base0 = smem_u32(stage_base);
+            const uint64_t da_hi0 = smem_desc(base0 + off_a_hi, a_lbo, a_sbo, a_lay);
+            const uint64_t db_hi0 = smem_desc(base0 + off_b_hi, b_lbo, b_sbo, b_lay);
+            const uint64_t da_lo0 = smem_desc(base0 + off_a_lo, a_lbo, a_sbo, a_lay);
+            const uint64_t db_lo0 = smem_desc(base0 + off_b_lo, b_lbo, b_sbo, b_lay);
+            const uint32_t a_kinc = a_kstep >> 4, b_kinc = b_kstep >> 4, stage_inc = (uint32_t)p.stage_bytes >> 4;
+            RingPos rp{0, 0};
+            uint32_t tile_i = 0;
             uint32_t overwrites[2] = {0, 0};        // how often each TMEM region has been restarted
             bool ok = true;
             for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++tile_i) {
                 int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
                 int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+                const uint32_t idesc = idesc0 | ((uint32_t)(tile_cols(p, nt) >> 3) << 17);
                 const uint32_t total_reg = tile_i & 1;
                 uint32_t reg = total_reg, d_tmem = 0;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const bool chunk_start = (kb % p.chunk_blocks) == 0;
+                int chunk_pos = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    const bool chunk_start = chunk_pos == 0;
                     if (chunk_start) {
                         // chunk 0 goes to the tile's total region, later chunks restart the other region
                         reg = (kb == 0) ? total_reg : (total_reg ^ 1);
@@ -309,20 +408,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         tc_fence_after();
                         d_tmem = tmem_base + reg * BN_MAX;
                     }
-                    const int s = it % p.stages;
-                    const uint32_t ph = (it / p.stages) & 1;
+                    const int s = rp.stage;
                     uint64_t* bar = p.split_pass ? &ctrl->ready[s] : &ctrl->full[s];
-                    if (!wait_bar(bar, ph, ctrl, p.status)) { ok = false; break; }
+                    if (!wait_bar(bar, rp.phase, ctrl, p.status)) { ok = false; break; }
+                    rp.advance(p.stages);
                     tc_fence_after();
-                    const uint32_t base = smem_u32(stage_base + (size_t)s * p.stage_bytes);
+                    const uint32_t soff = (uint32_t)s * stage_inc;
                     const int steps = (kb == nkb - 1) ? tail : BK / UMMA_K;
                     for (int ks = 0; ks < steps; ++ks) {
-                        const uint64_t a_hi = smem_desc(base + off_a_hi + ks * a_kstep, a_lbo, a_sbo, a_lay);
-                        const uint64_t b_hi = smem_desc(base + off_b_hi + ks * b_kstep, b_lbo, b_sbo, b_lay);
+                        const uint64_t a_hi = da_hi0 + (uint64_t)(soff + ks * a_kinc);
+                        const uint64_t b_hi = db_hi0 + (uint64_t)(soff + ks * b_kinc);
                         const uint32_t accumulate = (chunk_start && ks == 0) ? 0u : 1u;
                         if (p.three_x) {
-                            const uint64_t a_lo = smem_desc(base + off_a_lo + ks * a_kstep, a_lbo, a_sbo, a_lay);
-                            const uint64_t b_lo = smem_desc(base + off_b_lo + ks * b_kstep, b_lbo, b_sbo, b_lay);
+                            const uint64_t a_lo = da_lo0 + (uint64_t)(soff + ks * a_kinc);
+                            const uint64_t b_lo = db_lo0 + (uint64_t)(soff + ks * b_kinc);
                             umma_tf32(d_tmem, a_lo, b_hi, idesc, accumulate);
                             umma_tf32(d_tmem, a_hi, b_lo, idesc, 1u);
                             umma_tf32(d_tmem, a_hi, b_hi, idesc, 1u);
@@ -331,8 +430,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                     }
                     umma_commit(smem_u32(&ctrl->empty[s]));      // frees the stage when these products are done
-                    const bool chunk_end = ((kb + 1) % p.chunk_blocks) == 0 || kb == nkb - 1;
-                    if (chunk_end) umma_commit(smem_u32(&ctrl->reg_full[reg]));
+                    ++chunk_pos;
+                    if (chunk_pos == p.chunk_blocks || kb == nkb - 1) {
+                        umma_commit(smem_u32(&ctrl->reg_full[reg]));
+                        chunk_pos = 0;
+                    }
                 }
             }
         }
@@ -340,9 +442,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                         // TMEM lane quarter this warp may read
         const int ew = warp - 2;                        // 0..3, index of this warp among the epilogue warps
-        float* tr = epi_scratch + ew * (32 * 33);       // 32x32 staging tile of this warp (padded)
+        uint8_t* stg = epi_scratch + ew * (2 * EPI_STAGE_BYTES);     // two 32x32 store-staging blocks of this warp
+        const uint32_t lane_off = (uint32_t)(q * 32) << 16;
         const bool c_vec = ((((uintptr_t)d.C) & 15) == 0) && ((d.ldc & 3) == 0);
-        uint32_t tile_i = 0;
+        const bool bias_vec = (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) && ((((uintptr_t)d.bias) & 15) == 0);
+        const bool h_vec = (EPI == EPI_TANHP) && ((((uintptr_t)d.Hm) & 15) == 0) && ((d.ldh & 3) == 0);
+        uint32_t tile_i = 0, stg_i = 0;
         uint32_t reads[2] = {0, 0};             // how often each TMEM region has been waited for
         bool ok = true;
         for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++tile_i) {
@@ -350,6 +455,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int64_t kbeg_; int nkb_, tail_; unit_k_range(p, sp, kbeg_, nkb_, tail_);
             const int n_chunks = (nkb_ + p.chunk_blocks - 1) / p.chunk_blocks;
             const uint32_t acc = tile_i & 1, oth = acc ^ 1;
+            const int n0 = nt * p.bn;
+            const int chunks = (min(p.bn, (int)d.N - n0) + 31) >> 5;       // 32-column blocks of this tile inside the matrix
             if (!wait_bar(&ctrl->reg_full[acc], reads[acc] & 1, ctrl, p.status)) { ok = false; break; }
             reads[acc]++;
             tc_fence_after();
@@ -358,8 +465,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (!wait_bar(&ctrl->reg_full[oth], reads[oth] & 1, ctrl, p.status)) { ok = false; break; }
                 reads[oth]++;
                 tc_fence_after();
-                const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-                for (int c = 0; c < (p.bn + 31) / 32; ++c) {
+                for (int c = 0; c < chunks; ++c) {
                     uint32_t x[32], y[32];
                     tmem_ld32(tmem_base + oth * BN_MAX + c * 32 + lane_off, x);
                     tmem_ld32(tmem_base + acc * BN_MAX + c * 32 + lane_off, y);
@@ -374,130 +480,140 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->reg_free[oth]));
             }
             if (!ok) break;
-            const int64_t r = (int64_t)mt * BM + q * 32 + lane;
+            const int r0w = mt * BM + q * 32;                 // first row of this warp's 32-row block
+            const int64_t r = (int64_t)r0w + lane;
             const bool rv = r < d.M;
-            const int64_t n0 = (int64_t)nt * p.bn;
-            const int chunks = (p.bn + 31) / 32;
             float run_m = -INFINITY, run_s = 0.f, zl = 0.f;
-            int64_t lab = -1;
+            int lab = -1;
             bool have_zl = false;
-            if (EPI == EPI_LOGITS && rv) lab = (int64_t)__ldg(d.labels + r);
+            if (EPI == EPI_LOGITS && rv) lab = __ldg(d.labels + r);
             for (int c = 0; c < chunks; ++c) {
+                const int c0 = n0 + c * 32;
+                const int nvalid = min(32, (int)d.N - c0);      // < 32 only in the last block of a row of the matrix
+                const bool full = nvalid == 32;
                 uint32_t raw[32];
-                tmem_ld32(tmem_base + acc * BN_MAX + c * 32 + ((uint32_t)(q * 32) << 16), raw);
+                tmem_ld32(tmem_base + acc * BN_MAX + c * 32 + lane_off, raw);
                 tmem_ld_wait();
-                const int64_t c0 = n0 + c * 32;
-                int nvalid = (int)min((int64_t)32, min((int64_t)p.bn - c * 32, d.N - c0));
-                if (nvalid < 0) nvalid = 0;
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j]);
+                bool do_store = true;
 
                 if (EPI == EPI_SGEMM) {
-                    if (rv) {
-                        float* dst = d.C + r * d.ldc + c0;
-                        if (d.beta != 0.f) {
+                    if (d.beta != 0.f) {
+                        if (rv) {
+                            const float* src = d.C + r * d.ldc + c0;
+                            if (c_vec && full) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) if (j < nvalid) v[j] = fmaf(d.beta, dst[j], d.alpha * v[j]);
-                        } else {
+                                for (int j = 0; j < 32; j += 4) {
+                                    const float4 o = *reinterpret_cast<const float4*>(src + j);
+                                    v[j] = fmaf(d.beta, o.x, d.alpha * v[j]); v[j + 1] = fmaf(d.beta, o.y, d.alpha * v[j + 1]);
+                                    v[j + 2] = fmaf(d.beta, o.z, d.alpha * v[j + 2]); v[j + 3] = fmaf(d.beta, o.w, d.alpha * v[j + 3]);
+                                }
+                            } else {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] = d.alpha * v[j];
+                                for (int j = 0; j < 32; ++j) if (j < nvalid) v[j] = fmaf(d.beta, src[j], d.alpha * v[j]);
+                            }
                         }
-                        if (c_vec && nvalid == 32) {
+                    } else {
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        } else {
+                        for (int j = 0; j < 32; ++j) v[j] = d.alpha * v[j];
+                    }
+                } else if (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) {
+                    if (bias_vec && full) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 bb = __ldg(reinterpret_cast<const float4*>(d.bias + c0 + j));
+                            v[j] += bb.x; v[j + 1] += bb.y; v[j + 2] += bb.z; v[j + 3] += bb.w;
                         }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) if (j < nvalid) v[j] += __ldg(d.bias + c0 + j);
                     }
-                } else if (EPI == EPI_PARTIAL) {
-                    if (rv) {
-                        float* dst = d.partials + ((int64_t)sp * d.M + r) * d.ldp + c0;     // ldp % 4 == 0, base 256-aligned
-                        if (nvalid == 32) {
+                    if (EPI == EPI_BIAS_TANH) {
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        } else {
+                        for (int j = 0; j < 32; ++j) v[j] = tanhf(v[j]);
+                    } else {
+                        float cm = -INFINITY;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
-                        }
-                    }
-                } else if (EPI == EPI_BIAS_TANH) {
-                    if (rv) {
-                        float* dst = d.C + r * d.ldc + c0;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) if (j < nvalid) v[j] = tanhf(v[j] + __ldg(d.bias + c0 + j));
-                        if (c_vec && nvalid == 32) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
-                        }
-                    }
-                } else if (EPI == EPI_LOGITS) {
-                    float cm = -INFINITY;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        v[j] = (j < nvalid) ? v[j] + __ldg(d.bias + c0 + j) : -INFINITY;
-                        cm = fmaxf(cm, v[j]);
-                    }
-                    if (nvalid > 0) {
+                        for (int j = 0; j < 32; ++j) { if (j >= nvalid) v[j] = -INFINITY; cm = fmaxf(cm, v[j]); }
                         const float nm = fmaxf(run_m, cm);
                         float s = 0.f;
+                        if (full) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) if (j < nvalid) s += exp_mode(v[j] - nm, p.fast_math);
+                            for (int j = 0; j < 32; ++j) s += exp_mode(v[j] - nm, p.fast_math);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) if (j < nvalid) s += exp_mode(v[j] - nm, p.fast_math);
+                        }
                         run_s = (run_m == -INFINITY ? 0.f : run_s * exp_mode(run_m - nm, p.fast_math)) + s;
                         run_m = nm;
-                        if (rv) {
-                            if (lab >= c0 && lab < c0 + nvalid) {
+                        if ((unsigned)(lab - c0) < (unsigned)nvalid) {
 #pragma unroll
-                                for (int j = 0; j < 32; ++j) if (c0 + j == lab) zl = v[j];
-                                have_zl = true;
-                            }
-                            if (d.C) {
-                                float* dst = d.C + r * d.ldc + c0;
-                                if (c_vec && nvalid == 32) {
-#pragma unroll
-                                    for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                                } else {
-#pragma unroll
-                                    for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
-                                }
-                            }
+                            for (int j = 0; j < 32; ++j) if (c0 + j == lab) zl = v[j];
+                            have_zl = true;
                         }
+                        do_store = d.C != nullptr;
                     }
                 } else if (EPI == EPI_TANHP) {
                     if (rv) {
                         const float* hp = d.Hm + r * d.ldh + c0;
-                        float* dst = d.C + r * d.ldc + c0;
+                        if (h_vec && full) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (j < nvalid) { const float h = __ldg(hp + j); v[j] = (1.f - h * h) * v[j]; } else v[j] = 0.f;
-                        }
-                        if (c_vec && nvalid == 32) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            for (int j = 0; j < 32; j += 4) {
+                                const float4 h = __ldg(reinterpret_cast<const float4*>(hp + j));
+                                v[j] *= (1.f - h.x * h.x); v[j + 1] *= (1.f - h.y * h.y);
+                                v[j + 2] *= (1.f - h.z * h.z); v[j + 3] *= (1.f - h.w * h.w);
+                            }
                         } else {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
+                            for (int j = 0; j < 32; ++j) {
+                                if (j < nvalid) { const float h = __ldg(hp + j); v[j] = (1.f - h * h) * v[j]; } else v[j] = 0.f;
+                            }
                         }
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = 0.f;
                     }
-                    if (d.colsum_part) {
-                        // column sums of this warp's 32 rows, rows added in index order
+                }
+
+                // ---- store the 32x32 block
+                if (do_store) {
+                    if (p.c_tma) {
+                        uint8_t* blk = stg + (stg_i & 1) * EPI_STAGE_BYTES;
+                        ++stg_i;
+                        if (lane == 0) bulk_wait_read_1();      // the store issued from this block two blocks ago has been read
                         __syncwarp();
+                        // row `lane` of the block, 16-byte pieces XOR-swizzled with the row (128B swizzle)
+                        float4* rowp = reinterpret_cast<float4*>(blk + lane * 128);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) tr[lane * 33 + j] = v[j];
+                        for (int j = 0; j < 8; ++j)
+                            rowp[j ^ (lane & 7)] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        proxy_fence_async();
                         __syncwarp();
-                        float s = 0.f;
+                        if (lane == 0 && r0w < d.M) {
+                            tma_store_3d(&map_c, smem_u32(blk), c0, r0w, EPI == EPI_PARTIAL ? sp : 0);
+                            bulk_commit();
+                        }
+                    } else if (rv) {
+                        float* dst = (EPI == EPI_PARTIAL) ? d.partials + ((int64_t)sp * d.M + r) * d.ldp + c0
+                                                          : d.C + r * d.ldc + c0;
+                        if ((EPI == EPI_PARTIAL || c_vec) && full) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) s += tr[i * 33 + lane];
-                        // one partial row per 32-row group (4 per tile); the reduction kernel adds them in index order
-                        if (lane < nvalid) d.colsum_part[((int64_t)mt * 4 + q) * d.N + c0 + lane] = s;
+                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
+                        }
                     }
+                }
+                if (EPI == EPI_TANHP && d.colsum_part) {
+                    // column sums of this warp's 32 rows: one partial row per 32-row group (4 per tile); the
+                    // reduction kernel adds the groups in index order
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) if (j >= nvalid) v[j] = 0.f;
+                    const float s = warp_transpose_sum(v, lane);
+                    if (lane < nvalid) d.colsum_part[((int64_t)mt * 4 + q) * d.N + c0 + lane] = s;
                 }
             }
             // all TMEM reads of this accumulator stage are done: hand it back to the MMA warp
@@ -514,97 +630,94 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 for (int cc = 1; cc < d.ones_cols; ++cc) d.C[r * d.ldc + d.N + cc] = 0.f;
             }
         }
+        if (lane == 0) bulk_wait_all();         // every store of this warp has left shared memory and is complete
     } else if (p.split_pass) {
-        // ------------------------------------------------------------------ operand pass (hi/lo split, logits -> delta)
+        // ------------------------------------------------------------------ operand pass (lo parts, logits -> delta)
         const int st = threadIdx.x - (2 + NUM_EPI_WARPS) * 32;          // 0..255
         constexpr int NT = NUM_SPLIT_WARPS * 32;
-        uint32_t it = 0;
+        // Position of this thread's 16-byte pieces in the A tile (piece index st + 256*i, i = 0..3).
+        //  K-major: row (st>>3) + 32*i of the tile, the four floats run along K from k0 + 4*kch
+        //  MN-major: k row st>>3, the four floats run along M from m0 + 32*i + 4*mch
+        const int a_row = st >> 3;
+        const int kch = (st & 7) ^ (a_row & 7);
+        const int mch = ((((st & 7) >> 1) ^ (a_row & 3)) << 1) | (st & 1);
+        const int n_classes = (int)p.n_classes, n_patterns = (int)p.n_patterns;
+        RingPos rp{0, 0};
         bool ok = true;
         for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
             int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
-            const int64_t m0 = (int64_t)mt * BM;
-            for (int kb = 0; kb < nkb; ++kb, ++it) {
-                const int s = it % p.stages;
-                const uint32_t ph = (it / p.stages) & 1;
-                if (!wait_bar(&ctrl->full[s], ph, ctrl, p.status)) { ok = false; break; }
+            const int m0 = mt * BM;
+            const int b_cols = tile_cols(p, nt);
+            // K-major logits (the pattern is the row): statistics of this thread's four rows, once per tile
+            float row_lse[4] = {0.f, 0.f, 0.f, 0.f};
+            int row_lab[4] = {-1, -1, -1, -1};
+            if (d.a_transform && !p.a_mn) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int pat = m0 + a_row + 32 * i;
+                    if (pat < n_patterns) { row_lse[i] = __ldg(d.lse + pat); row_lab[i] = __ldg(d.labels + pat); }
+                }
+            }
+            int k0 = (int)kbeg;
+            for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
+                const int s = rp.stage;
+                // MN-major logits (the pattern is the k row): statistics of this thread's pattern in this block
+                float k_lse = 0.f; int k_lab = -1;
+                const int kpat = k0 + a_row;
+                if (d.a_transform && p.a_mn && kpat < n_patterns) { k_lse = __ldg(d.lse + kpat); k_lab = __ldg(d.labels + kpat); }
+                if (!wait_bar(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
+                rp.advance(p.stages);
                 uint8_t* base = stage_base + (size_t)s * p.stage_bytes;
-                const int64_t k0 = kbeg + (int64_t)kb * BK;
-                // A tile: 1024 float4
                 float4* a_hi = reinterpret_cast<float4*>(base + off_a_hi);
                 float4* a_lo = reinterpret_cast<float4*>(base + off_a_lo);
+                if (d.a_transform) {
 #pragma unroll
-                for (int i = 0; i < (BM * BK / 4) / NT; ++i) {
-                    const int idx = st + NT * i;
-                    float4 x = a_hi[idx];
-                    if (d.a_transform) {
-                        // un-swizzle the position of this 16-byte chunk to (pattern, class)
-                        int64_t pat, cls;
+                    for (int i = 0; i < (BM * BK / 4) / NT; ++i) {
+                        const int idx = st + NT * i;
+                        float4 x = a_hi[idx];
                         if (!p.a_mn) {
-                            const int row = idx >> 3, ch = (idx & 7) ^ (row & 7);
-                            pat = d.a_pattern_is_m ? m0 + row : k0 + ch * 4;
-                            cls = d.a_pattern_is_m ? k0 + ch * 4 : m0 + row;
-                            // K-major: the four elements run along K
-                            if (d.a_pattern_is_m) {
-                                if (pat < p.n_patterns) {
-                                    const float l = __ldg(d.lse + pat); const int64_t lb = (int64_t)__ldg(d.labels + pat);
-                                    x.x = (cls + 0 < p.n_classes) ? exp_mode(x.x - l, p.fast_math) - (cls + 0 == lb ? 1.f : 0.f) : 0.f;
-                                    x.y = (cls + 1 < p.n_classes) ? exp_mode(x.y - l, p.fast_math) - (cls + 1 == lb ? 1.f : 0.f) : 0.f;
-                                    x.z = (cls + 2 < p.n_classes) ? exp_mode(x.z - l, p.fast_math) - (cls + 2 == lb ? 1.f : 0.f) : 0.f;
-                                    x.w = (cls + 3 < p.n_classes) ? exp_mode(x.w - l, p.fast_math) - (cls + 3 == lb ? 1.f : 0.f) : 0.f;
-                                } else x = make_float4(0.f, 0.f, 0.f, 0.f);
-                            } else {
-                                float e[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-                                for (int t = 0; t < 4; ++t) {
-                                    const int64_t pp = pat + t;
-                                    if (pp < p.n_patterns && cls < p.n_classes)
-                                        e[t] = exp_mode(e[t] - __ldg(d.lse + pp), p.fast_math) - (cls == (int64_t)__ldg(d.labels + pp) ? 1.f : 0.f);
-                                    else e[t] = 0.f;
-                                }
-                                x = make_float4(e[0], e[1], e[2], e[3]);
-                            }
+                            const int cls = k0 + kch * 4;
+                            if (m0 + a_row + 32 * i < n_patterns) {
+                                x.x = delta_of(x.x, row_lse[i], cls + 0, row_lab[i], n_classes, p.fast_math);
+                                x.y = delta_of(x.y, row_lse[i], cls + 1, row_lab[i], n_classes, p.fast_math);
+                                x.z = delta_of(x.z, row_lse[i], cls + 2, row_lab[i], n_classes, p.fast_math);
+                                x.w = delta_of(x.w, row_lse[i], cls + 3, row_lab[i], n_classes, p.fast_math);
+                            } else x = make_float4(0.f, 0.f, 0.f, 0.f);
                         } else {
-                            // 32-byte units of a 128-byte row are XORed with (row & 3); a float4 is half a unit
-                            const int g = idx >> 8, krow = (idx & 255) >> 3;
-                            const int ch = ((((idx & 7) >> 1) ^ (krow & 3)) << 1) | (idx & 1);
-                            const int64_t mn = m0 + g * 32 + ch * 4, kk = k0 + krow;
-                            // MN-major: the four elements run along M
-                            if (d.a_pattern_is_m) {
-                                float e[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-                                for (int t = 0; t < 4; ++t) {
-                                    const int64_t pp = mn + t;
-                                    if (pp < p.n_patterns && kk < p.n_classes)
-                                        e[t] = exp_mode(e[t] - __ldg(d.lse + pp), p.fast_math) - (kk == (int64_t)__ldg(d.labels + pp) ? 1.f : 0.f);
-                                    else e[t] = 0.f;
-                                }
-                                x = make_float4(e[0], e[1], e[2], e[3]);
-                            } else {
-                                pat = kk; cls = mn;
-                                if (pat < p.n_patterns) {
-                                    const float l = __ldg(d.lse + pat); const int64_t lb = (int64_t)__ldg(d.labels + pat);
-                                    x.x = (cls + 0 < p.n_classes) ? exp_mode(x.x - l, p.fast_math) - (cls + 0 == lb ? 1.f : 0.f) : 0.f;
-                                    x.y = (cls + 1 < p.n_classes) ? exp_mode(x.y - l, p.fast_math) - (cls + 1 == lb ? 1.f : 0.f) : 0.f;
-                                    x.z = (cls + 2 < p.n_classes) ? exp_mode(x.z - l, p.fast_math) - (cls + 2 == lb ? 1.f : 0.f) : 0.f;
-                                    x.w = (cls + 3 < p.n_classes) ? exp_mode(x.w - l, p.fast_math) - (cls + 3 == lb ? 1.f : 0.f) : 0.f;
-                                } else x = make_float4(0.f, 0.f, 0.f, 0.f);
-                            }
+                            const int cls = m0 + 32 * i + mch * 4;
+                            if (kpat < n_patterns) {
+                                x.x = delta_of(x.x, k_lse, cls + 0, k_lab, n_classes, p.fast_math);
+                                x.y = delta_of(x.y, k_lse, cls + 1, k_lab, n_classes, p.fast_math);
+                                x.z = delta_of(x.z, k_lse, cls + 2, k_lab, n_classes, p.fast_math);
+                                x.w = delta_of(x.w, k_lse, cls + 3, k_lab, n_classes, p.fast_math);
+                            } else x = make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                        if (p.three_x) {
+                            float4 h, l; split4(x, p.round_hi, h, l);
+                            a_hi[idx] = h; a_lo[idx] = l;
+                        } else {
+                            a_hi[idx] = x;
                         }
                     }
-                    const float4 h = make_float4(to_tf32(x.x), to_tf32(x.y), to_tf32(x.z), to_tf32(x.w));
-                    a_hi[idx] = h;
-                    if (p.three_x) a_lo[idx] = make_float4(to_tf32(x.x - h.x), to_tf32(x.y - h.y), to_tf32(x.z - h.z), to_tf32(x.w - h.w));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < (BM * BK / 4) / NT; ++i) {
+                        const int idx = st + NT * i;
+                        float4 h, l; split4(a_hi[idx], p.round_hi, h, l);
+                        if (p.round_hi) a_hi[idx] = h;
+                        a_lo[idx] = l;
+                    }
                 }
                 if (p.three_x) {
                     float4* b_hi = reinterpret_cast<float4*>(base + off_b_hi);
                     float4* b_lo = reinterpret_cast<float4*>(base + off_b_lo);
-                    const int nvec = p.b_tile_bytes / 16;
+                    const int nvec = b_cols * 8;                 // 128 bytes per column of the tile
+#pragma unroll 4
                     for (int idx = st; idx < nvec; idx += NT) {
-                        const float4 x = b_hi[idx];
-                        const float4 h = make_float4(to_tf32(x.x), to_tf32(x.y), to_tf32(x.z), to_tf32(x.w));
-                        b_hi[idx] = h;
-                        b_lo[idx] = make_float4(to_tf32(x.x - h.x), to_tf32(x.y - h.y), to_tf32(x.z - h.z), to_tf32(x.w - h.w));
+                        float4 h, l; split4(b_hi[idx], p.round_hi, h, l);
+                        if (p.round_hi) b_hi[idx] = h;
+                        b_lo[idx] = l;
                     }
                 }
                 proxy_fence_async();            // make these generic-proxy writes visible to the tensor core's reads
@@ -660,6 +773,20 @@ bool make_map(CUtensorMap* map, const float* base, int64_t inner, int64_t outer,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of an output written with TMA stores: `slices` matrices of `rows` x `cols` floats, rows `ld` floats
+// apart, one after the other; box = one 32 x 32 block (128-byte rows, 128B swizzle).  Stores are clipped at the
+// edges of the matrix (rows exactly, columns at the next multiple of four).
+bool make_store_map(CUtensorMap* map, const float* base, int64_t cols, int64_t rows, int64_t ld, int64_t slices) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)slices};
+    cuuint64_t gstride[2] = {(cuuint64_t)ld * sizeof(float), (cuuint64_t)rows * (cuuint64_t)ld * sizeof(float)};
+    cuuint32_t box[3] = {32, 32, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool operand_ok(const float* base, int64_t s_major, int64_t s_minor_is_one_other) {
     (void)s_minor_is_one_other;
     return (((uintptr_t)base) & 15) == 0 && (s_major & 3) == 0 && s_major >= 4 && s_major < ((int64_t)1 << 38);
@@ -682,14 +809,15 @@ int* status_ptr() {
 }
 
 template <int EPI>
-ulsnn_status_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
+ulsnn_status_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const TcParams& p, int smem_bytes, int grid,
+                      cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
             return ULSNN_ERR_CUDA;
         configured = true;
     }
-    tc_gemm_kernel<EPI><<<grid, NUM_THREADS, smem_bytes, stream>>>(ma, mb, p);
+    tc_gemm_kernel<EPI><<<grid, NUM_THREADS, smem_bytes, stream>>>(ma, mb, mc, p);
     count_launch(1);
     return cuda_ok(cudaGetLastError());
 }
@@ -700,12 +828,9 @@ int tc_tile_m() { return BM; }
 int tc_colsum_groups() { return 4; }
 
 int tc_tile_n(const GemmDesc& d) {
-    const bool b_mn = !(d.b_sk == 1);                     // B(k,j): contiguous along j unless contiguous along k
-    const int gran = b_mn ? 32 : 16;
-    const int64_t tiles = (d.N + BN_MAX - 1) / BN_MAX;
-    int64_t bn = (d.N + tiles - 1) / tiles;
-    bn = (bn + gran - 1) / gran * gran;
-    if (bn < gran) bn = gran;
+    // 32-column blocks are the unit of the epilogue's stores; tiles are as wide as TMEM allows and the last one
+    // of a row is given to the tensor core at its own, smaller width
+    int64_t bn = (d.N + 31) / 32 * 32;
     if (bn > BN_MAX) bn = BN_MAX;
     return (int)bn;
 }
@@ -719,6 +844,8 @@ bool tc_gemm_supported(const GemmDesc& d) {
     if (!b_k && d.b_sn != 1) return false;
     if (!operand_ok(d.A, a_k ? d.a_sm : d.a_sk, 0)) return false;
     if (!operand_ok(d.B, b_k ? d.b_sn : d.b_sk, 0)) return false;
+    // logits as the A operand: either [pattern x class] read K-major or its transpose read MN-major
+    if (d.a_transform && (a_k != (d.a_pattern_is_m != 0))) return false;
     return true;
 }
 
@@ -729,6 +856,7 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.a_mn = (d.a_sk == 1) ? 0 : 1;
     p.b_mn = (d.b_sk == 1) ? 0 : 1;
     p.bn = tc_tile_n(d);
+    p.n_gran = p.b_mn ? 32 : 16;
     p.tiles_m = (int)((d.M + BM - 1) / BM);
     p.tiles_n = (int)((d.N + p.bn - 1) / p.bn);
     const int splits = (d.epi == EPI_PARTIAL) ? d.splits : 1;
@@ -739,6 +867,7 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.split_pass = (three_x || d.a_transform) ? 1 : 0;
     p.fast_math = three_x ? 0 : 1;
     p.chunk_blocks = three_x ? 8 : (1 << 30);       // 256 elements of K per accumulator in the accurate mode
+    p.round_hi = 1;
     p.b_tile_bytes = p.bn * 128;
     p.stage_bytes = (A_TILE_BYTES + p.b_tile_bytes) * (three_x ? 2 : 1);
     int stages = (SMEM_BUDGET - 1024 - EPI_SCRATCH_BYTES - CTRL_BYTES) / p.stage_bytes;
@@ -757,14 +886,27 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     const bool okb = p.b_mn ? make_map(&mb, d.B, d.N, d.K, d.b_sk, 32, 32, true) : make_map(&mb, d.B, d.K, d.N, d.b_sn, 32, p.bn, false);
     if (!oka || !okb) return ULSNN_ERR_CUDA;
 
+    // the output goes through TMA stores when its rows are 16-byte aligned; otherwise the epilogue stores directly
+    CUtensorMap mc;
+    memset(&mc, 0, sizeof(mc));
+    if (d.epi == EPI_PARTIAL) {
+        p.c_tma = make_store_map(&mc, d.partials, d.N, d.M, d.ldp, splits) ? 1 : 0;
+    } else if (d.C && (((uintptr_t)d.C) & 15) == 0 && (d.ldc & 3) == 0 && d.ldc >= 4) {
+        // A TMA store clips a row at the next 16-byte boundary past the matrix edge, so a width that is not a multiple
+        // of four spills up to three floats into the row's padding.  That padding is scratch in the library's own
+        // logit and delta buffers; it belongs to the caller in C, and it is the ones column in an activation buffer.
+        const bool pad_is_scratch = d.epi == EPI_LOGITS || d.epi == EPI_TANHP;
+        if ((d.N & 3) == 0 || pad_is_scratch) p.c_tma = make_store_map(&mc, d.C, d.N, d.M, d.ldc, 1) ? 1 : 0;
+    }
+
     const int smem_bytes = 1024 + stages * p.stage_bytes + EPI_SCRATCH_BYTES + CTRL_BYTES;
     const int grid = p.units < sm_count() ? p.units : sm_count();
     switch (d.epi) {
-        case EPI_SGEMM:     return launch<EPI_SGEMM>(ma, mb, p, smem_bytes, grid, stream);
-        case EPI_BIAS_TANH: return launch<EPI_BIAS_TANH>(ma, mb, p, smem_bytes, grid, stream);
-        case EPI_LOGITS:    return launch<EPI_LOGITS>(ma, mb, p, smem_bytes, grid, stream);
-        case EPI_TANHP:     return launch<EPI_TANHP>(ma, mb, p, smem_bytes, grid, stream);
-        case EPI_PARTIAL:   return launch<EPI_PARTIAL>(ma, mb, p, smem_bytes, grid, stream);
+        case EPI_SGEMM:     return launch<EPI_SGEMM>(ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_BIAS_TANH: return launch<EPI_BIAS_TANH>(ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_LOGITS:    return launch<EPI_LOGITS>(ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_TANHP:     return launch<EPI_TANHP>(ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_PARTIAL:   return launch<EPI_PARTIAL>(ma, mb, mc, p, smem_bytes, grid, stream);
     }
     return ULSNN_ERR_INVALID_ARG;
 }
