@@ -149,10 +149,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Round to the nearest TF32 value (10 mantissa bits), ties away from zero, as cvt.rna.tf32.f32 does, but with two
+// integer instructions at full rate: the conversion instruction runs at a fraction of it, and the operand pass
+// applies this to every element of every landed tile.
 __device__ __forceinline__ float to_tf32(float x) {
-    uint32_t u;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
-    return __uint_as_float(u);
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
 }
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
