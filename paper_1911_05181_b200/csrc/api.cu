@@ -55,11 +55,11 @@ struct SplitPlan { int splits; int64_t k_per_split; };
 
 // Fixed by the shapes only.  Slices are at most SLICE_CAP long once K is large (bounds the fp32 rounding of a
 // long sum), and short-and-wide products get enough slices to fill the GPU.
-SplitPlan plan_splits(int64_t tiles, int64_t K) {
+SplitPlan plan_splits(int64_t tiles, int64_t K, int64_t slots) {
     int64_t s_acc = (K > 2 * SLICE_CAP) ? (K + SLICE_CAP - 1) / SLICE_CAP : 1;
     int64_t s_fill = 1;
-    if (tiles < 148 && K >= 1024) {
-        s_fill = (296 + tiles - 1) / tiles;
+    if (tiles < slots && K >= 1024) {
+        s_fill = (2 * slots + tiles - 1) / tiles;
         if (s_fill > K / 512) s_fill = K / 512;
         if (s_fill < 1) s_fill = 1;
     }
@@ -71,8 +71,10 @@ SplitPlan plan_splits(int64_t tiles, int64_t K) {
     return SplitPlan{(int)s, kps};
 }
 
+int64_t slots_of(const GemmDesc& d, bool tc) { return tc ? tc_slots(d) : simt_slots(); }
+
 int64_t tiles_of(const GemmDesc& d, bool tc) {
-    const int64_t bm = tc ? tc_tile_m() : simt_tile_m();
+    const int64_t bm = tc ? tc_tile_m(d) : simt_tile_m();
     const int64_t bn = tc ? tc_tile_n(d) : simt_tile_n();
     return ((d.M + bm - 1) / bm) * ((d.N + bn - 1) / bn);
 }
@@ -104,7 +106,7 @@ GemmDesc sgemm_desc(const SgemmArgs& a) {
 }
 
 size_t sgemm_ws_for(const GemmDesc& d, bool tc) {
-    const SplitPlan p = plan_splits(tiles_of(d, tc), d.K);
+    const SplitPlan p = plan_splits(tiles_of(d, tc), d.K, slots_of(d, tc));
     if (p.splits <= 1) return 0;
     return align256((size_t)p.splits * (size_t)d.M * (size_t)round_up(d.N, 4) * sizeof(float));
 }
@@ -119,7 +121,7 @@ ulsnn_status_t sgemm_impl(const SgemmArgs& a, ulsnn_math_t math, void* ws, size_
     if (!a.A || !a.B) return ULSNN_ERR_INVALID_ARG;
     GemmDesc d = sgemm_desc(a);
     const bool tc = use_tc(d, math);
-    const SplitPlan p = plan_splits(tiles_of(d, tc), d.K);
+    const SplitPlan p = plan_splits(tiles_of(d, tc), d.K, slots_of(d, tc));
     if (p.splits <= 1) return run_gemm(d, math, stream);
     const int64_t ldp = round_up(d.N, 4);
     const size_t need = (size_t)p.splits * (size_t)d.M * (size_t)ldp * sizeof(float);
@@ -321,9 +323,9 @@ size_t wgrad_partial_bound(const int32_t* sizes, int w, int64_t B) {
     const int64_t ldp = round_up(d.N, 4);
     int64_t smax = (B + SLICE_CAP - 1) / SLICE_CAP;
     for (int tc = 0; tc < 2; ++tc) {
-        const int64_t tiles = tiles_of(d, tc != 0);
-        if (tiles < 148 && B >= 1024) {
-            int64_t f = (296 + tiles - 1) / tiles;
+        const int64_t tiles = tiles_of(d, tc != 0), slots = slots_of(d, tc != 0);
+        if (tiles < slots && B >= 1024) {
+            int64_t f = (2 * slots + tiles - 1) / tiles;
             if (f > B / 512) f = B / 512;
             if (f > smax) smax = f;
         }
@@ -566,7 +568,8 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
         if (w >= 1) { d.B = h->H[w]; d.b_sk = h->ldh[w]; } else { d.B = X; d.b_sk = ldx; }
         d.b_sn = 1;
         d.alpha = 1.f; d.beta = 0.f; d.epi = EPI_PARTIAL;
-        const SplitPlan p = plan_splits(tiles_of(d, use_tc(d, h->math)), d.K);
+        const bool tc = use_tc(d, h->math);
+        const SplitPlan p = plan_splits(tiles_of(d, tc), d.K, slots_of(d, tc));
         d.splits = p.splits; d.k_per_split = p.k_per_split;
         d.ldp = round_up(d.N, 4); d.partials = h->partials;
         if ((size_t)p.splits * (size_t)d.M * (size_t)d.ldp * sizeof(float) > h->partials_bytes) return ULSNN_ERR_WORKSPACE_TOO_SMALL;

@@ -51,8 +51,11 @@ int simt_tile_n();
 // tcgen05 engine (tc_gemm.cu).  tc_gemm_supported: can TMA address these operands (16-byte aligned bases, leading
 // dimensions that are multiples of 4 floats)?  tc_tile_n: the column-tile width it will use for this product.
 bool tc_gemm_supported(const GemmDesc& d);
-int tc_tile_m();
+int tc_tile_m(const GemmDesc& d);
 int tc_tile_n(const GemmDesc& d);
+// how many tiles each engine works on at a time (CTAs, or CTA pairs): what a split-K plan has to fill
+int tc_slots(const GemmDesc& d);
+int simt_slots();
 // EPI_TANHP writes this many partial column-sum rows per 128-row tile (row index = tile*groups + group)
 int tc_colsum_groups();
 int simt_colsum_groups();

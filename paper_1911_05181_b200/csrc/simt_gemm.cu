@@ -221,6 +221,7 @@ ulsnn_status_t launch(const GemmDesc& d, cudaStream_t stream) {
 
 int simt_tile_m() { return BM; }
 int simt_tile_n() { return BN; }
+int simt_slots() { return 148; }
 int simt_colsum_groups() { return 1; }
 
 ulsnn_status_t simt_gemm_launch(const GemmDesc& d, cudaStream_t stream) {

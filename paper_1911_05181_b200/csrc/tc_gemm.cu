@@ -45,6 +45,7 @@ constexpr int NUM_SPLIT_WARPS = 8;
 constexpr int NUM_WARPS = 2 + NUM_EPI_WARPS + NUM_SPLIT_WARPS;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 8;
+constexpr int NUM_SMS = 148;               // B200; fixes the tile schedule (and with it every summation order)
 constexpr int A_TILE_BYTES = BM * BK * 4;                       // 16 KB
 constexpr int SMEM_BUDGET = 227 * 1024;
 constexpr int EPI_STAGE_BYTES = 32 * 128;                        // one 32x32 fp32 block, 128B-swizzled
@@ -56,15 +57,16 @@ struct TcParams {
     GemmDesc d;
     int bn;                 // column-tile width, a multiple of 32 (the last tile of a row may use fewer columns)
     int n_gran;             // granularity of the width the tensor core is given for that last tile: 16, or 32 when B is MN-major
-    int tiles_m, tiles_n;
+    int tiles_m, tiles_n;   // tiles_m counts tiles of 128*CG rows
     int units;              // tiles_m * tiles_n * splits
     int stages;
-    int b_tile_bytes;       // bn * 128
+    int b_tile_bytes;       // bytes of one CTA's B tile: (bn / CG) * 128
     int stage_bytes;
     int three_x, a_mn, b_mn, split_pass;
     int chunk_blocks;       // k-blocks accumulated on one TMEM accumulator before it is added into the tile total
     int fast_math;          // TF32 mode: approximate exp
     int round_hi;           // 3xTF32: the operand pass also rewrites the landed tile as hi = tf32_rn(x) (lo = x - hi)
+    int ready_arrivals;     // arrivals per CTA on a stage's `ready` barrier (operand-pass warps, or one relay)
     int c_tma;              // the output (C or the split-K partials) is written with TMA stores
     int64_t n_patterns, n_classes;      // bounds of the logits operand when a_transform
     int* status;
@@ -82,11 +84,27 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// arrive on the barrier at the same shared-memory offset in CTA 0 of the cluster (which may be this CTA)
+__device__ __forceinline__ void mbar_arrive_rank0(uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, 0;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
@@ -103,27 +121,50 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+// CG = number of CTAs (1 or 2) that share one tile: with 2, one tcgen05.mma spans the tensor cores of both SMs of
+// a cluster, each CTA holding its 128 rows of A, its half of the B tile and its 128 rows of the accumulator
+template <int CG> __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    if constexpr (CG == 1) asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    else asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
 }
-__device__ __forceinline__ void tmem_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+template <int CG> __device__ __forceinline__ void tmem_relinquish() {
+    if constexpr (CG == 1) asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    else asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+template <int CG> __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    if constexpr (CG == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void proxy_fence_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+template <int CG>
 __device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    if constexpr (CG == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    }
 }
+// The barrier (at this offset in every CTA of the tile) gets one arrival when the products issued so far are done.
+template <int CG>
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if constexpr (CG == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}"
+            ::"r"(bar) : "memory");
+    }
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -291,7 +332,7 @@ __device__ __forceinline__ void split4(const float4 x, bool round_hi, float4& hi
     }
 }
 
-template <int EPI>
+template <int EPI, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, const TcParams p) {
@@ -304,26 +345,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const GemmDesc& d = p.d;
+    // With CG == 2 the two CTAs of a cluster work on the same sequence of tiles.  CTA 0 issues the products; the
+    // `ready` and `reg_free` barriers that its issuing thread waits on live in CTA 0 and collect arrivals from both.
+    const int rank = (CG == 2) ? (int)cluster_ctarank() : 0;
+    const int first_unit = blockIdx.x / CG, unit_step = gridDim.x / CG;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&ctrl->full[s]), 1);
-            mbar_init(smem_u32(&ctrl->ready[s]), NUM_SPLIT_WARPS);
+            mbar_init(smem_u32(&ctrl->ready[s]), CG * p.ready_arrivals);
             mbar_init(smem_u32(&ctrl->empty[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&ctrl->reg_full[a]), 1);
-            mbar_init(smem_u32(&ctrl->reg_free[a]), NUM_EPI_WARPS);
+            mbar_init(smem_u32(&ctrl->reg_free[a]), CG * NUM_EPI_WARPS);
         }
         ctrl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&ctrl->tmem_base), 512);
-        tmem_relinquish();
+        tmem_alloc<CG>(smem_u32(&ctrl->tmem_base), 512);
+        tmem_relinquish<CG>();
     }
     tc_fence_before();
-    __syncthreads();
+    if constexpr (CG == 2) cluster_sync_all(); else __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
 
@@ -336,13 +381,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
             RingPos rp{0, 0};
             bool ok = true;
-            for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
+            for (int u = first_unit; u < p.units && ok; u += unit_step) {
                 int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
                 int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
-                const int m0 = mt * BM, n0 = nt * p.bn;
-                // a K-major B tile is one box of bn rows (rows past the matrix arrive as zeros); an MN-major one is a
-                // box per 32 columns, and only the boxes the products read are fetched
-                const int b_boxes = tile_cols(p, nt) >> 5;
+                // this CTA's rows of A and its share of the tile's columns of B
+                const int b_cols = tile_cols(p, nt) / CG;
+                const int m0 = (mt * CG + rank) * BM, n0 = nt * p.bn + rank * b_cols;
+                // a K-major B tile is one box of bn/CG rows (rows past the matrix arrive as zeros); an MN-major one is
+                // a box per 32 columns, and only the boxes the products read are fetched
+                const int b_boxes = b_cols >> 5;
                 const uint32_t tx_bytes = (uint32_t)(A_TILE_BYTES + (p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes));
                 int k0 = (int)kbeg;
                 for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
@@ -371,9 +418,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             const uint32_t idesc0 = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
-                                    ((uint32_t)(BM >> 4) << 24);
+                                    ((uint32_t)((BM * CG) >> 4) << 24);
             // K-major (128B swizzle): 8-row groups 1024 B apart (SBO), K advance = 32 B inside the swizzled row.
             // MN-major (128B swizzle, 32-byte atoms): 32-element groups BK*128 B apart (LBO), 4-k groups 512 B apart
             // (SBO), K advance = 8 rows = 1024 B.
@@ -392,7 +439,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t tile_i = 0;
             uint32_t overwrites[2] = {0, 0};        // how often each TMEM region has been restarted
             bool ok = true;
-            for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++tile_i) {
+            for (int u = first_unit; u < p.units && ok; u += unit_step, ++tile_i) {
                 int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
                 int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
                 const uint32_t idesc = idesc0 | ((uint32_t)(tile_cols(p, nt) >> 3) << 17);
@@ -410,7 +457,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         d_tmem = tmem_base + reg * BN_MAX;
                     }
                     const int s = rp.stage;
-                    uint64_t* bar = p.split_pass ? &ctrl->ready[s] : &ctrl->full[s];
+                    uint64_t* bar = (CG == 2 || p.split_pass) ? &ctrl->ready[s] : &ctrl->full[s];
                     if (!wait_bar(bar, rp.phase, ctrl, p.status)) { ok = false; break; }
                     rp.advance(p.stages);
                     tc_fence_after();
@@ -423,17 +470,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         if (p.three_x) {
                             const uint64_t a_lo = da_lo0 + (uint64_t)(soff + ks * a_kinc);
                             const uint64_t b_lo = db_lo0 + (uint64_t)(soff + ks * b_kinc);
-                            umma_tf32(d_tmem, a_lo, b_hi, idesc, accumulate);
-                            umma_tf32(d_tmem, a_hi, b_lo, idesc, 1u);
-                            umma_tf32(d_tmem, a_hi, b_hi, idesc, 1u);
+                            umma_tf32<CG>(d_tmem, a_lo, b_hi, idesc, accumulate);
+                            umma_tf32<CG>(d_tmem, a_hi, b_lo, idesc, 1u);
+                            umma_tf32<CG>(d_tmem, a_hi, b_hi, idesc, 1u);
                         } else {
-                            umma_tf32(d_tmem, a_hi, b_hi, idesc, accumulate);
+                            umma_tf32<CG>(d_tmem, a_hi, b_hi, idesc, accumulate);
                         }
                     }
-                    umma_commit(smem_u32(&ctrl->empty[s]));      // frees the stage when these products are done
+                    umma_commit<CG>(smem_u32(&ctrl->empty[s]));      // frees the stage (in every CTA of the tile) when these products are done
                     ++chunk_pos;
                     if (chunk_pos == p.chunk_blocks || kb == nkb - 1) {
-                        umma_commit(smem_u32(&ctrl->reg_full[reg]));
+                        umma_commit<CG>(smem_u32(&ctrl->reg_full[reg]));
                         chunk_pos = 0;
                     }
                 }
@@ -451,7 +498,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t tile_i = 0, stg_i = 0;
         uint32_t reads[2] = {0, 0};             // how often each TMEM region has been waited for
         bool ok = true;
-        for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++tile_i) {
+        for (int u = first_unit; u < p.units && ok; u += unit_step, ++tile_i) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
             int64_t kbeg_; int nkb_, tail_; unit_k_range(p, sp, kbeg_, nkb_, tail_);
             const int n_chunks = (nkb_ + p.chunk_blocks - 1) / p.chunk_blocks;
@@ -478,10 +525,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->reg_free[oth]));
+                if (lane == 0) { if constexpr (CG == 2) mbar_arrive_rank0(smem_u32(&ctrl->reg_free[oth])); else mbar_arrive(smem_u32(&ctrl->reg_free[oth])); }
             }
             if (!ok) break;
-            const int r0w = mt * BM + q * 32;                 // first row of this warp's 32-row block
+            const int r0w = (mt * CG + rank) * BM + q * 32;   // first row of this warp's 32-row block
             const int64_t r = (int64_t)r0w + lane;
             const bool rv = r < d.M;
             float run_m = -INFINITY, run_s = 0.f, zl = 0.f;
@@ -614,13 +661,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 32; ++j) if (j >= nvalid) v[j] = 0.f;
                     const float s = warp_transpose_sum(v, lane);
-                    if (lane < nvalid) d.colsum_part[((int64_t)mt * 4 + q) * d.N + c0 + lane] = s;
+                    if (lane < nvalid) d.colsum_part[((int64_t)(mt * CG + rank) * 4 + q) * d.N + c0 + lane] = s;
                 }
             }
             // all TMEM reads of this accumulator stage are done: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl->reg_free[acc]));
+            if (lane == 0) { if constexpr (CG == 2) mbar_arrive_rank0(smem_u32(&ctrl->reg_free[acc])); else mbar_arrive(smem_u32(&ctrl->reg_free[acc])); }
 
             if (EPI == EPI_LOGITS && rv) {
                 d.stats[r * d.stats_ld + nt] = make_float2(run_m, run_s);
@@ -645,11 +692,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int n_classes = (int)p.n_classes, n_patterns = (int)p.n_patterns;
         RingPos rp{0, 0};
         bool ok = true;
-        for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
+        for (int u = first_unit; u < p.units && ok; u += unit_step) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
             int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
-            const int m0 = mt * BM;
-            const int b_cols = tile_cols(p, nt);
+            const int m0 = (mt * CG + rank) * BM;
+            const int b_cols = tile_cols(p, nt) / CG;
             // K-major logits (the pattern is the row): statistics of this thread's four rows, once per tile
             float row_lse[4] = {0.f, 0.f, 0.f, 0.f};
             int row_lab[4] = {-1, -1, -1, -1};
@@ -723,7 +770,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 proxy_fence_async();            // make these generic-proxy writes visible to the tensor core's reads
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->ready[s]));
+                if (lane == 0) { if constexpr (CG == 2) mbar_arrive_rank0(smem_u32(&ctrl->ready[s])); else mbar_arrive(smem_u32(&ctrl->ready[s])); }
+            }
+        }
+    } else if (CG == 2 && warp == 2 + NUM_EPI_WARPS) {
+        // ------------------------------------------------------------------ no operand pass: tell CTA 0 when a stage of this CTA has landed
+        if (lane == 0) {
+            RingPos rp{0, 0};
+            bool ok = true;
+            for (int u = first_unit; u < p.units && ok; u += unit_step) {
+                int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
+                int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+                for (int kb = 0; kb < nkb; ++kb) {
+                    const int s = rp.stage;
+                    if (!wait_bar(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
+                    rp.advance(p.stages);
+                    mbar_arrive_rank0(smem_u32(&ctrl->ready[s]));
+                }
             }
         }
     }
@@ -733,11 +796,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // give copies that may still be in flight time to land before the shared memory is released
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
     }
+    __syncwarp();
     tc_fence_before();
-    __syncthreads();
+    // nobody leaves while the other CTA of the tile may still signal a barrier here or read this CTA's operands
+    if constexpr (CG == 2) cluster_sync_all(); else __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 512);
+        tmem_dealloc<CG>(tmem_base, 512);
     }
 }
 
@@ -809,29 +874,52 @@ int* status_ptr() {
     return ptr;
 }
 
-template <int EPI>
+template <int EPI, int CG>
 ulsnn_status_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const TcParams& p, int smem_bytes, int grid,
                       cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
+        if (cudaFuncSetAttribute(tc_gemm_kernel<EPI, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
             return ULSNN_ERR_CUDA;
         configured = true;
     }
-    tc_gemm_kernel<EPI><<<grid, NUM_THREADS, smem_bytes, stream>>>(ma, mb, mc, p);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG>, ma, mb, mc, p);
     count_launch(1);
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(e == cudaSuccess ? cudaGetLastError() : e);
+}
+
+template <int EPI>
+ulsnn_status_t launch_cg(int cg, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const TcParams& p, int smem_bytes,
+                         int grid, cudaStream_t stream) {
+    return cg == 2 ? launch<EPI, 2>(ma, mb, mc, p, smem_bytes, grid, stream) : launch<EPI, 1>(ma, mb, mc, p, smem_bytes, grid, stream);
 }
 
 }  // namespace
 
-int tc_tile_m() { return BM; }
+// Products with more than one 128-row tile are computed by pairs of CTAs (256-row tiles, tcgen05 cta_group::2):
+// per product instruction each SM then reads half as much of B from its shared memory.
+int tc_cta_group(const GemmDesc& d) { return d.M > BM ? 2 : 1; }
+int tc_tile_m(const GemmDesc& d) { return BM * tc_cta_group(d); }
+int tc_slots(const GemmDesc& d) { return NUM_SMS / tc_cta_group(d); }
 int tc_colsum_groups() { return 4; }
 
 int tc_tile_n(const GemmDesc& d) {
-    // 32-column blocks are the unit of the epilogue's stores; tiles are as wide as TMEM allows and the last one
-    // of a row is given to the tensor core at its own, smaller width
-    int64_t bn = (d.N + 31) / 32 * 32;
+    // 32-column blocks are the unit of the epilogue's stores (64 where two CTAs each fetch 32-column boxes of an
+    // MN-major B); tiles are as wide as TMEM allows and the last one of a row is given to the tensor core at its
+    // own, smaller width
+    const bool b_mn = !(d.b_sk == 1);
+    const int64_t g = (b_mn && tc_cta_group(d) == 2) ? 64 : 32;
+    int64_t bn = (d.N + g - 1) / g * g;
     if (bn > BN_MAX) bn = BN_MAX;
     return (int)bn;
 }
@@ -856,9 +944,10 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.d = d;
     p.a_mn = (d.a_sk == 1) ? 0 : 1;
     p.b_mn = (d.b_sk == 1) ? 0 : 1;
+    const int cg = tc_cta_group(d);
     p.bn = tc_tile_n(d);
-    p.n_gran = p.b_mn ? 32 : 16;
-    p.tiles_m = (int)((d.M + BM - 1) / BM);
+    p.n_gran = cg * (p.b_mn ? 32 : 16);
+    p.tiles_m = (int)((d.M + BM * cg - 1) / (BM * cg));
     p.tiles_n = (int)((d.N + p.bn - 1) / p.bn);
     const int splits = (d.epi == EPI_PARTIAL) ? d.splits : 1;
     const int64_t units = (int64_t)p.tiles_m * p.tiles_n * splits;
@@ -866,10 +955,11 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.units = (int)units;
     p.three_x = three_x ? 1 : 0;
     p.split_pass = (three_x || d.a_transform) ? 1 : 0;
+    p.ready_arrivals = p.split_pass ? NUM_SPLIT_WARPS : 1;
     p.fast_math = three_x ? 0 : 1;
     p.chunk_blocks = three_x ? 8 : (1 << 30);       // 256 elements of K per accumulator in the accurate mode
     p.round_hi = 1;
-    p.b_tile_bytes = p.bn * 128;
+    p.b_tile_bytes = (p.bn / cg) * 128;
     p.stage_bytes = (A_TILE_BYTES + p.b_tile_bytes) * (three_x ? 2 : 1);
     int stages = (SMEM_BUDGET - 1024 - EPI_SCRATCH_BYTES - CTRL_BYTES) / p.stage_bytes;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -884,7 +974,7 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
 
     CUtensorMap ma, mb;
     const bool oka = p.a_mn ? make_map(&ma, d.A, d.M, d.K, d.a_sk, 32, 32, true) : make_map(&ma, d.A, d.K, d.M, d.a_sm, 32, BM, false);
-    const bool okb = p.b_mn ? make_map(&mb, d.B, d.N, d.K, d.b_sk, 32, 32, true) : make_map(&mb, d.B, d.K, d.N, d.b_sn, 32, p.bn, false);
+    const bool okb = p.b_mn ? make_map(&mb, d.B, d.N, d.K, d.b_sk, 32, 32, true) : make_map(&mb, d.B, d.K, d.N, d.b_sn, 32, p.bn / cg, false);
     if (!oka || !okb) return ULSNN_ERR_CUDA;
 
     // the output goes through TMA stores when its rows are 16-byte aligned; otherwise the epilogue stores directly
@@ -901,13 +991,14 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     }
 
     const int smem_bytes = 1024 + stages * p.stage_bytes + EPI_SCRATCH_BYTES + CTRL_BYTES;
-    const int grid = p.units < sm_count() ? p.units : sm_count();
+    const int slots = sm_count() / cg;
+    const int grid = cg * (p.units < slots ? p.units : slots);
     switch (d.epi) {
-        case EPI_SGEMM:     return launch<EPI_SGEMM>(ma, mb, mc, p, smem_bytes, grid, stream);
-        case EPI_BIAS_TANH: return launch<EPI_BIAS_TANH>(ma, mb, mc, p, smem_bytes, grid, stream);
-        case EPI_LOGITS:    return launch<EPI_LOGITS>(ma, mb, mc, p, smem_bytes, grid, stream);
-        case EPI_TANHP:     return launch<EPI_TANHP>(ma, mb, mc, p, smem_bytes, grid, stream);
-        case EPI_PARTIAL:   return launch<EPI_PARTIAL>(ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_SGEMM:     return launch_cg<EPI_SGEMM>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_BIAS_TANH: return launch_cg<EPI_BIAS_TANH>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_LOGITS:    return launch_cg<EPI_LOGITS>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_TANHP:     return launch_cg<EPI_TANHP>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_PARTIAL:   return launch_cg<EPI_PARTIAL>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
     }
     return ULSNN_ERR_INVALID_ARG;
 }
