@@ -29,6 +29,7 @@
 #include <math.h>
 #include <string.h>
 #include <mutex>
+#include <type_traits>
 
 namespace ulsnn {
 
@@ -65,7 +66,6 @@ struct TcParams {
     int three_x, a_mn, b_mn, split_pass;
     int chunk_blocks;       // k-blocks accumulated on one TMEM accumulator before it is added into the tile total
     int fast_math;          // TF32 mode: approximate exp
-    int round_hi;           // 3xTF32: the operand pass also rewrites the landed tile as hi = tf32_rn(x) (lo = x - hi)
     int ready_arrivals;     // arrivals per CTA on a stage's `ready` barrier (operand-pass warps, or one relay)
     int c_tma;              // the output (C or the split-K partials) is written with TMA stores
     int64_t n_patterns, n_classes;      // bounds of the logits operand when a_transform
@@ -83,6 +83,14 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// One lane of a converged warp (always the same one for the full mask).  The warps that issue TMA copies and
+// tensor-core products run their loops with all 32 lanes and elect the issuing lane around the instruction
+// itself: addresses and descriptors then stay warp-uniform values.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred = 0;
+    asm volatile("{\n\t.reg .pred px;\n\telect.sync _|px, 0xffffffff;\n\t@px mov.s32 %0, 1;\n\t}" : "+r"(pred));
+    return pred != 0;
 }
 // arrive on the barrier at the same shared-memory offset in CTA 0 of the cluster (which may be this CTA)
 __device__ __forceinline__ void mbar_arrive_rank0(uint32_t bar) {
@@ -140,30 +148,34 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void proxy_fence_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 template <int CG>
 __device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    if constexpr (CG == 1) {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    if (elect_one()) {
+        if constexpr (CG == 1) {
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "setp.ne.b32 p, %4, 0;\n\t"
+                "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+                ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+        } else {
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "setp.ne.b32 p, %4, 0;\n\t"
+                "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+                ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+        }
     }
 }
 // The barrier (at this offset in every CTA of the tile) gets one arrival when the products issued so far are done.
 template <int CG>
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-    if constexpr (CG == 1) {
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
-            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}"
-            ::"r"(bar) : "memory");
+    if (elect_one()) {
+        if constexpr (CG == 1) {
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+        } else {
+            asm volatile(
+                "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+                "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}"
+                ::"r"(bar) : "memory");
+        }
     }
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -210,7 +222,7 @@ __device__ __forceinline__ float exp_fast_accurate(float x) {
     const float p = ex2_approx(th);
     return fmaf(p, tl * 0.693147180559945f, p);
 }
-__device__ __forceinline__ float exp_mode(float x, int fast) { return fast ? __expf(x) : exp_fast_accurate(x); }
+template <bool FAST> __device__ __forceinline__ float exp_t(float x) { return FAST ? __expf(x) : exp_fast_accurate(x); }
 
 // Shared-memory matrix descriptor of a swizzled tile (sm_100 format: version 1 at bit 46; layout type at bits
 // 61-63: 2 = 128B swizzle of 16-byte units, 1 = 128B swizzle of 32-byte units).
@@ -246,6 +258,12 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctrl* c
         }
     }
     return true;
+}
+
+// wait_bar by all lanes of a converged warp, with one outcome for the warp
+__device__ __forceinline__ bool wait_bar_warp(uint64_t* bar, uint32_t parity, Ctrl* ctrl, int* status) {
+    const bool ok = wait_bar(bar, parity, ctrl, status);
+    return __all_sync(0xffffffffu, ok);
 }
 
 __device__ __forceinline__ void unit_coords(const TcParams& p, int u, int& mt, int& nt, int& sp) {
@@ -313,23 +331,19 @@ __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
 }
 
 // softmax(z) - onehot from a stored logit: e = exp(z - lse) - [cls == label], 0 outside the matrix
-__device__ __forceinline__ float delta_of(float z, float lse, int cls, int label, int n_classes, int fast) {
-    return (cls < n_classes) ? exp_mode(z - lse, fast) - (cls == label ? 1.f : 0.f) : 0.f;
+template <bool FAST>
+__device__ __forceinline__ float delta_of(float z, float lse, int cls, int label, int n_classes) {
+    const float e = exp_t<FAST>(z - lse) - (cls == label ? 1.f : 0.f);
+    return cls < n_classes ? e : 0.f;
 }
 
-__device__ __forceinline__ float lo_part(float x) {
-    return to_tf32(x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u));
-}
-// hi/lo parts of four values: with round_hi the hi part is rounded to nearest and has to be written back,
-// otherwise it is the truncation the tensor core applies to the stored word by itself
-__device__ __forceinline__ void split4(const float4 x, bool round_hi, float4& hi, float4& lo) {
-    if (round_hi) {
-        hi = make_float4(to_tf32(x.x), to_tf32(x.y), to_tf32(x.z), to_tf32(x.w));
-        lo = make_float4(to_tf32(x.x - hi.x), to_tf32(x.y - hi.y), to_tf32(x.z - hi.z), to_tf32(x.w - hi.w));
-    } else {
-        hi = x;
-        lo = make_float4(lo_part(x.x), lo_part(x.y), lo_part(x.z), lo_part(x.w));
-    }
+// hi = tf32_rn(x), lo = tf32_rn(x - hi).  (The tensor core ignores the low 13 mantissa bits of a stored word, so the
+// landed tile could serve as hi = trunc(x) without being rewritten; but then every lo has the sign of its x, the
+// truncation of the accumulator no longer averages out over the lo products, and the measured error of the
+// weight gradients was 2.4 times larger.)
+__device__ __forceinline__ void split4(const float4 x, float4& hi, float4& lo) {
+    hi = make_float4(to_tf32(x.x), to_tf32(x.y), to_tf32(x.z), to_tf32(x.w));
+    lo = make_float4(to_tf32(x.x - hi.x), to_tf32(x.y - hi.y), to_tf32(x.z - hi.z), to_tf32(x.w - hi.w));
 }
 
 template <int EPI, int CG>
@@ -378,28 +392,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            RingPos rp{0, 0};
-            bool ok = true;
-            for (int u = first_unit; u < p.units && ok; u += unit_step) {
-                int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-                int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
-                // this CTA's rows of A and its share of the tile's columns of B
-                const int b_cols = tile_cols(p, nt) / CG;
-                const int m0 = (mt * CG + rank) * BM, n0 = nt * p.bn + rank * b_cols;
-                // a K-major B tile is one box of bn/CG rows (rows past the matrix arrive as zeros); an MN-major one is
-                // a box per 32 columns, and only the boxes the products read are fetched
-                const int b_boxes = b_cols >> 5;
-                const uint32_t tx_bytes = (uint32_t)(A_TILE_BYTES + (p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes));
-                int k0 = (int)kbeg;
-                for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
-                    const int s = rp.stage;
-                    if (!wait_bar(&ctrl->empty[s], rp.phase ^ 1, ctrl, p.status)) { ok = false; break; }
-                    rp.advance(p.stages);
-                    const uint32_t bar = smem_u32(&ctrl->full[s]);
+        RingPos rp{0, 0};
+        bool ok = true;
+        for (int u = first_unit; u < p.units && ok; u += unit_step) {
+            int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
+            int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+            // this CTA's rows of A and its share of the tile's columns of B
+            const int b_cols = tile_cols(p, nt) / CG;
+            const int m0 = (mt * CG + rank) * BM, n0 = nt * p.bn + rank * b_cols;
+            // a K-major B tile is one box of bn/CG rows (rows past the matrix arrive as zeros); an MN-major one is
+            // a box per 32 columns, and only the boxes the products read are fetched
+            const int b_boxes = b_cols >> 5;
+            const uint32_t tx_bytes = (uint32_t)(A_TILE_BYTES + (p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes));
+            int k0 = (int)kbeg;
+            for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
+                const int s = rp.stage;
+                if (!wait_bar_warp(&ctrl->empty[s], rp.phase ^ 1, ctrl, p.status)) { ok = false; break; }
+                rp.advance(p.stages);
+                const uint32_t bar = smem_u32(&ctrl->full[s]);
+                const uint32_t sa = smem_u32(stage_base + (size_t)s * p.stage_bytes + off_a_hi);
+                const uint32_t sb = sa + off_b_hi;
+                if (elect_one()) {
                     mbar_expect_tx(bar, tx_bytes);
-                    const uint32_t sa = smem_u32(stage_base + (size_t)s * p.stage_bytes + off_a_hi);
-                    const uint32_t sb = sa + off_b_hi;
                     if (!p.a_mn) {
                         tma_load_2d(sa, &map_a, k0, m0, bar);                       // box {32 k, 128 rows}
                     } else {
@@ -408,17 +422,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             tma_load_2d(sa + g * (BK * 128), &map_a, m0 + 32 * g, k0, bar);
                     }
                     if (!p.b_mn) {
-                        tma_load_2d(sb, &map_b, k0, n0, bar);                       // box {32 k, bn rows}
+                        tma_load_2d(sb, &map_b, k0, n0, bar);                       // box {32 k, bn/CG rows}
                     } else {
-                        for (int g = 0; g < b_boxes; ++g)
-                            tma_load_2d(sb + g * (BK * 128), &map_b, n0 + 32 * g, k0, bar);
+#pragma unroll
+                        for (int g = 0; g < BN_MAX / 32; ++g)
+                            if (g < b_boxes) tma_load_2d(sb + g * (BK * 128), &map_b, n0 + 32 * g, k0, bar);
                     }
                 }
+                __syncwarp();
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0 && rank == 0) {
+        if (rank == 0) {
             const uint32_t idesc0 = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
                                     ((uint32_t)((BM * CG) >> 4) << 24);
             // K-major (128B swizzle): 8-row groups 1024 B apart (SBO), K advance = 32 B inside the swizzled row.
@@ -451,19 +467,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (chunk_start) {
                         // chunk 0 goes to the tile's total region, later chunks restart the other region
                         reg = (kb == 0) ? total_reg : (total_reg ^ 1);
-                        if (!wait_bar(&ctrl->reg_free[reg], (overwrites[reg] & 1) ^ 1, ctrl, p.status)) { ok = false; break; }
+                        if (!wait_bar_warp(&ctrl->reg_free[reg], (overwrites[reg] & 1) ^ 1, ctrl, p.status)) { ok = false; break; }
                         overwrites[reg]++;
                         tc_fence_after();
                         d_tmem = tmem_base + reg * BN_MAX;
                     }
                     const int s = rp.stage;
                     uint64_t* bar = (CG == 2 || p.split_pass) ? &ctrl->ready[s] : &ctrl->full[s];
-                    if (!wait_bar(bar, rp.phase, ctrl, p.status)) { ok = false; break; }
+                    if (!wait_bar_warp(bar, rp.phase, ctrl, p.status)) { ok = false; break; }
                     rp.advance(p.stages);
                     tc_fence_after();
                     const uint32_t soff = (uint32_t)s * stage_inc;
                     const int steps = (kb == nkb - 1) ? tail : BK / UMMA_K;
-                    for (int ks = 0; ks < steps; ++ks) {
+#pragma unroll
+                    for (int ks = 0; ks < BK / UMMA_K; ++ks) {
+                        if (ks >= steps) break;
                         const uint64_t a_hi = da_hi0 + (uint64_t)(soff + ks * a_kinc);
                         const uint64_t b_hi = db_hi0 + (uint64_t)(soff + ks * b_kinc);
                         const uint32_t accumulate = (chunk_start && ks == 0) ? 0u : 1u;
@@ -587,14 +605,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int j = 0; j < 32; ++j) { if (j >= nvalid) v[j] = -INFINITY; cm = fmaxf(cm, v[j]); }
                         const float nm = fmaxf(run_m, cm);
                         float s = 0.f;
-                        if (full) {
+                        auto sum_exp = [&](auto fast_tag) {
+                            constexpr bool FAST = decltype(fast_tag)::value;
+                            if (full) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) s += exp_mode(v[j] - nm, p.fast_math);
-                        } else {
+                                for (int j = 0; j < 32; ++j) s += exp_t<FAST>(v[j] - nm);
+                            } else {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) if (j < nvalid) s += exp_mode(v[j] - nm, p.fast_math);
-                        }
-                        run_s = (run_m == -INFINITY ? 0.f : run_s * exp_mode(run_m - nm, p.fast_math)) + s;
+                                for (int j = 0; j < 32; ++j) if (j < nvalid) s += exp_t<FAST>(v[j] - nm);
+                            }
+                            run_s = (run_m == -INFINITY ? 0.f : run_s * exp_t<FAST>(run_m - nm)) + s;
+                        };
+                        if (p.fast_math) sum_exp(std::true_type{}); else sum_exp(std::false_type{});
                         run_m = nm;
                         if ((unsigned)(lab - c0) < (unsigned)nvalid) {
 #pragma unroll
@@ -719,55 +741,59 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 uint8_t* base = stage_base + (size_t)s * p.stage_bytes;
                 float4* a_hi = reinterpret_cast<float4*>(base + off_a_hi);
                 float4* a_lo = reinterpret_cast<float4*>(base + off_a_lo);
-                if (d.a_transform) {
+                float4* b_hi = reinterpret_cast<float4*>(base + off_b_hi);
+                float4* b_lo = reinterpret_cast<float4*>(base + off_b_lo);
+                // The body is instantiated per (approximate exp?, 3xTF32?) so that its unrolled loops are straight-line code.
+                auto pass = [&](auto fast_tag, auto three_tag) {
+                    constexpr bool FAST = decltype(fast_tag)::value, THREE = decltype(three_tag)::value;
+                    constexpr int NA = (BM * BK / 4) / NT;          // 16-byte pieces of the A tile per thread
+                    float4 x[NA];
 #pragma unroll
-                    for (int i = 0; i < (BM * BK / 4) / NT; ++i) {
-                        const int idx = st + NT * i;
-                        float4 x = a_hi[idx];
+                    for (int i = 0; i < NA; ++i) x[i] = a_hi[st + NT * i];
+                    if (d.a_transform) {
                         if (!p.a_mn) {
                             const int cls = k0 + kch * 4;
-                            if (m0 + a_row + 32 * i < n_patterns) {
-                                x.x = delta_of(x.x, row_lse[i], cls + 0, row_lab[i], n_classes, p.fast_math);
-                                x.y = delta_of(x.y, row_lse[i], cls + 1, row_lab[i], n_classes, p.fast_math);
-                                x.z = delta_of(x.z, row_lse[i], cls + 2, row_lab[i], n_classes, p.fast_math);
-                                x.w = delta_of(x.w, row_lse[i], cls + 3, row_lab[i], n_classes, p.fast_math);
-                            } else x = make_float4(0.f, 0.f, 0.f, 0.f);
-                        } else {
-                            const int cls = m0 + 32 * i + mch * 4;
-                            if (kpat < n_patterns) {
-                                x.x = delta_of(x.x, k_lse, cls + 0, k_lab, n_classes, p.fast_math);
-                                x.y = delta_of(x.y, k_lse, cls + 1, k_lab, n_classes, p.fast_math);
-                                x.z = delta_of(x.z, k_lse, cls + 2, k_lab, n_classes, p.fast_math);
-                                x.w = delta_of(x.w, k_lse, cls + 3, k_lab, n_classes, p.fast_math);
-                            } else x = make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-                        if (p.three_x) {
-                            float4 h, l; split4(x, p.round_hi, h, l);
-                            a_hi[idx] = h; a_lo[idx] = l;
-                        } else {
-                            a_hi[idx] = x;
-                        }
-                    }
-                } else {
 #pragma unroll
-                    for (int i = 0; i < (BM * BK / 4) / NT; ++i) {
-                        const int idx = st + NT * i;
-                        float4 h, l; split4(a_hi[idx], p.round_hi, h, l);
-                        if (p.round_hi) a_hi[idx] = h;
-                        a_lo[idx] = l;
+                            for (int i = 0; i < NA; ++i) {
+                                const bool live = m0 + a_row + 32 * i < n_patterns;
+                                x[i].x = live ? delta_of<FAST>(x[i].x, row_lse[i], cls + 0, row_lab[i], n_classes) : 0.f;
+                                x[i].y = live ? delta_of<FAST>(x[i].y, row_lse[i], cls + 1, row_lab[i], n_classes) : 0.f;
+                                x[i].z = live ? delta_of<FAST>(x[i].z, row_lse[i], cls + 2, row_lab[i], n_classes) : 0.f;
+                                x[i].w = live ? delta_of<FAST>(x[i].w, row_lse[i], cls + 3, row_lab[i], n_classes) : 0.f;
+                            }
+                        } else {
+                            const bool live = kpat < n_patterns;
+#pragma unroll
+                            for (int i = 0; i < NA; ++i) {
+                                const int cls = m0 + 32 * i + mch * 4;
+                                x[i].x = live ? delta_of<FAST>(x[i].x, k_lse, cls + 0, k_lab, n_classes) : 0.f;
+                                x[i].y = live ? delta_of<FAST>(x[i].y, k_lse, cls + 1, k_lab, n_classes) : 0.f;
+                                x[i].z = live ? delta_of<FAST>(x[i].z, k_lse, cls + 2, k_lab, n_classes) : 0.f;
+                                x[i].w = live ? delta_of<FAST>(x[i].w, k_lse, cls + 3, k_lab, n_classes) : 0.f;
+                            }
+                        }
                     }
-                }
-                if (p.three_x) {
-                    float4* b_hi = reinterpret_cast<float4*>(base + off_b_hi);
-                    float4* b_lo = reinterpret_cast<float4*>(base + off_b_lo);
-                    const int nvec = b_cols * 8;                 // 128 bytes per column of the tile
+#pragma unroll
+                    for (int i = 0; i < NA; ++i) {
+                        if constexpr (THREE) {
+                            float4 h, l; split4(x[i], h, l);
+                            a_hi[st + NT * i] = h; a_lo[st + NT * i] = l;
+                        } else {
+                            a_hi[st + NT * i] = x[i];       // only reached when A was transformed
+                        }
+                    }
+                    if constexpr (THREE) {
+                        const int nvec = b_cols * 8;                 // 128 bytes per column of the tile
 #pragma unroll 4
-                    for (int idx = st; idx < nvec; idx += NT) {
-                        float4 h, l; split4(b_hi[idx], p.round_hi, h, l);
-                        if (p.round_hi) b_hi[idx] = h;
-                        b_lo[idx] = l;
+                        for (int idx = st; idx < nvec; idx += NT) {
+                            float4 h, l; split4(b_hi[idx], h, l);
+                            b_hi[idx] = h; b_lo[idx] = l;
+                        }
                     }
-                }
+                };
+                if (p.three_x) pass(std::false_type{}, std::true_type{});
+                else if (p.fast_math) pass(std::true_type{}, std::false_type{});
+                else pass(std::false_type{}, std::false_type{});
                 proxy_fence_async();            // make these generic-proxy writes visible to the tensor core's reads
                 __syncwarp();
                 if (lane == 0) { if constexpr (CG == 2) mbar_arrive_rank0(smem_u32(&ctrl->ready[s])); else mbar_arrive(smem_u32(&ctrl->ready[s])); }
@@ -775,18 +801,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if (CG == 2 && warp == 2 + NUM_EPI_WARPS) {
         // ------------------------------------------------------------------ no operand pass: tell CTA 0 when a stage of this CTA has landed
-        if (lane == 0) {
-            RingPos rp{0, 0};
-            bool ok = true;
-            for (int u = first_unit; u < p.units && ok; u += unit_step) {
-                int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-                int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
-                for (int kb = 0; kb < nkb; ++kb) {
-                    const int s = rp.stage;
-                    if (!wait_bar(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
-                    rp.advance(p.stages);
-                    mbar_arrive_rank0(smem_u32(&ctrl->ready[s]));
-                }
+        RingPos rp{0, 0};
+        bool ok = true;
+        for (int u = first_unit; u < p.units && ok; u += unit_step) {
+            int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
+            int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = rp.stage;
+                if (!wait_bar_warp(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
+                rp.advance(p.stages);
+                if (lane == 0) mbar_arrive_rank0(smem_u32(&ctrl->ready[s]));
             }
         }
     }
@@ -958,7 +982,6 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.ready_arrivals = p.split_pass ? NUM_SPLIT_WARPS : 1;
     p.fast_math = three_x ? 0 : 1;
     p.chunk_blocks = three_x ? 8 : (1 << 30);       // 256 elements of K per accumulator in the accurate mode
-    p.round_hi = 1;
     p.b_tile_bytes = (p.bn / cg) * 128;
     p.stage_bytes = (A_TILE_BYTES + p.b_tile_bytes) * (three_x ? 2 : 1);
     int stages = (SMEM_BUDGET - 1024 - EPI_SCRATCH_BYTES - CTRL_BYTES) / p.stage_bytes;
