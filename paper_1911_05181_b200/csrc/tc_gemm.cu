@@ -66,7 +66,6 @@ struct TcParams {
     int three_x, a_mn, b_mn, split_pass;
     int chunk_blocks;       // k-blocks accumulated on one TMEM accumulator before it is added into the tile total
     int fast_math;          // TF32 mode: approximate exp
-    int ready_arrivals;     // arrivals per CTA on a stage's `ready` barrier (operand-pass warps, or one relay)
     int c_tma;              // the output (C or the split-K partials) is written with TMA stores
     int64_t n_patterns, n_classes;      // bounds of the logits operand when a_transform
     int* status;
@@ -359,15 +358,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const GemmDesc& d = p.d;
-    // With CG == 2 the two CTAs of a cluster work on the same sequence of tiles.  CTA 0 issues the products; the
-    // `ready` and `reg_free` barriers that its issuing thread waits on live in CTA 0 and collect arrivals from both.
+    // With CG == 2 the two CTAs of a cluster work on the same sequence of tiles.  CTA 0 issues the products.  Its
+    // `ready` barriers collect its own operand-pass warps and one arrival per stage that warp 1 of CTA 1 sends over
+    // when CTA 1's stage is ready (an arrival on another CTA's barrier costs its sender about a microsecond, so it
+    // is kept off the warps that do the work); its `reg_free` barriers collect the epilogue warps of both CTAs.
     const int rank = (CG == 2) ? (int)cluster_ctarank() : 0;
     const int first_unit = blockIdx.x / CG, unit_step = gridDim.x / CG;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&ctrl->full[s]), 1);
-            mbar_init(smem_u32(&ctrl->ready[s]), CG * p.ready_arrivals);
+            // CTA 0: its own operand-pass warps plus one arrival relayed from CTA 1; CTA 1: its operand-pass warps
+            const int ready_count = (p.split_pass ? NUM_SPLIT_WARPS : 0) + ((CG == 2 && rank == 0) ? 1 : 0);
+            mbar_init(smem_u32(&ctrl->ready[s]), ready_count > 0 ? ready_count : 1);      // unused when nothing arrives on it
             mbar_init(smem_u32(&ctrl->empty[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -473,8 +476,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         d_tmem = tmem_base + reg * BN_MAX;
                     }
                     const int s = rp.stage;
-                    uint64_t* bar = (CG == 2 || p.split_pass) ? &ctrl->ready[s] : &ctrl->full[s];
-                    if (!wait_bar_warp(bar, rp.phase, ctrl, p.status)) { ok = false; break; }
+                    if (!p.split_pass && !wait_bar_warp(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
+                    if ((p.split_pass || CG == 2) && !wait_bar_warp(&ctrl->ready[s], rp.phase, ctrl, p.status)) { ok = false; break; }
                     rp.advance(p.stages);
                     tc_fence_after();
                     const uint32_t soff = (uint32_t)s * stage_inc;
@@ -501,6 +504,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         umma_commit<CG>(smem_u32(&ctrl->reg_full[reg]));
                         chunk_pos = 0;
                     }
+                }
+            }
+        }
+        if (CG == 2 && rank == 1) {
+            // CTA 1 issues nothing: this warp tells CTA 0 when a stage of CTA 1 is ready for the products
+            RingPos rp{0, 0};
+            bool ok = true;
+            for (int u = first_unit; u < p.units && ok; u += unit_step) {
+                int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
+                int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+                for (int kb = 0; kb < nkb; ++kb) {
+                    const int s = rp.stage;
+                    uint64_t* bar = p.split_pass ? &ctrl->ready[s] : &ctrl->full[s];
+                    if (!wait_bar_warp(bar, rp.phase, ctrl, p.status)) { ok = false; break; }
+                    rp.advance(p.stages);
+                    if (lane == 0) mbar_arrive_rank0(smem_u32(&ctrl->ready[s]));
+                    __syncwarp();
                 }
             }
         }
@@ -796,21 +816,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 else pass(std::false_type{}, std::false_type{});
                 proxy_fence_async();            // make these generic-proxy writes visible to the tensor core's reads
                 __syncwarp();
-                if (lane == 0) { if constexpr (CG == 2) mbar_arrive_rank0(smem_u32(&ctrl->ready[s])); else mbar_arrive(smem_u32(&ctrl->ready[s])); }
-            }
-        }
-    } else if (CG == 2 && warp == 2 + NUM_EPI_WARPS) {
-        // ------------------------------------------------------------------ no operand pass: tell CTA 0 when a stage of this CTA has landed
-        RingPos rp{0, 0};
-        bool ok = true;
-        for (int u = first_unit; u < p.units && ok; u += unit_step) {
-            int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-            int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = rp.stage;
-                if (!wait_bar_warp(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
-                rp.advance(p.stages);
-                if (lane == 0) mbar_arrive_rank0(smem_u32(&ctrl->ready[s]));
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->ready[s]));
             }
         }
     }
@@ -979,7 +985,6 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.units = (int)units;
     p.three_x = three_x ? 1 : 0;
     p.split_pass = (three_x || d.a_transform) ? 1 : 0;
-    p.ready_arrivals = p.split_pass ? NUM_SPLIT_WARPS : 1;
     p.fast_math = three_x ? 0 : 1;
     p.chunk_blocks = three_x ? 8 : (1 << 30);       // 256 elements of K per accumulator in the accurate mode
     p.b_tile_bytes = (p.bn / cg) * 128;
