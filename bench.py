@@ -65,7 +65,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -159,7 +159,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--math", default="3xtf32", choices=sorted(MATH))
@@ -322,7 +322,8 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "%s: %s MLP, %d patterns per GPU, seed %d" % (args.workload, "-".join(map(str, sizes)), batch, seed),
                    "math": args.math, "global_batch": batch * world, "parallelism": "dp%d" % world,
-                   "l2": "inputs and intermediates (X 105 MB, logits 840 MB per step) exceed the 126 MB L2; no flush",
+                   "l2": "no flush: inputs and intermediates of a step (X %.0f MB, logits %.0f MB) exceed the 126 MB L2"
+                         % (batch * sizes[0] * 4 / 1e6, batch * sizes[-1] * 4 / 1e6),
                    "step": "gradient evaluation + W -= lr*grad, lr = 1e-3 / global_batch"},
         "patterns_per_s": batch * world / (ms_step * 1e-3),
         "pct_of_tf32_peak": None,

@@ -27,14 +27,25 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ parts, int splits
     }
 }
 
-__global__ void colsum_reduce_kernel(const float* __restrict__ parts, int64_t tiles, int64_t N, int accumulate,
-                                     float* __restrict__ out) {
-    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= N) return;
+// out[j] = sum_t parts[t*N + j]: a block owns 32 columns; its 32 row lanes each add every 32nd partial row in
+// index order (double), then the 32 lane sums are added in lane order.  The order depends on (tiles, N) only.
+constexpr int CS_COLS = 32, CS_LANES = 32;
+__global__ void __launch_bounds__(CS_COLS * CS_LANES)
+colsum_reduce_kernel(const float* __restrict__ parts, int64_t tiles, int64_t N, int accumulate, float* __restrict__ out) {
+    __shared__ double red[CS_LANES][CS_COLS + 1];
+    const int tx = threadIdx.x % CS_COLS, ty = threadIdx.x / CS_COLS;
+    const int64_t j = (int64_t)blockIdx.x * CS_COLS + tx;
     double s = 0.0;
-    for (int64_t t = 0; t < tiles; ++t) s += (double)parts[t * N + j];
-    if (accumulate) s += (double)out[j];
-    out[j] = (float)s;
+    if (j < N) for (int64_t t = ty; t < tiles; t += CS_LANES) s += (double)parts[t * N + j];
+    red[ty][tx] = s;
+    __syncthreads();
+    if (ty == 0 && j < N) {
+        double tot = 0.0;
+#pragma unroll
+        for (int l = 0; l < CS_LANES; ++l) tot += red[l][tx];
+        if (accumulate) tot += (double)out[j];
+        out[j] = (float)tot;
+    }
 }
 
 constexpr int RS_THREADS = 256;
@@ -155,7 +166,7 @@ ulsnn_status_t launch_splitk_reduce(const float* parts, int splits, int64_t M, i
 ulsnn_status_t launch_colsum_reduce(const float* parts, int64_t tiles, int64_t N, int accumulate, float* out,
                                     cudaStream_t stream) {
     if (N <= 0) return ULSNN_OK;
-    colsum_reduce_kernel<<<(unsigned)((N + 127) / 128), 128, 0, stream>>>(parts, tiles, N, accumulate, out);
+    colsum_reduce_kernel<<<(unsigned)((N + CS_COLS - 1) / CS_COLS), CS_COLS * CS_LANES, 0, stream>>>(parts, tiles, N, accumulate, out);
     ulsnn::count_launch(2);
     return cuda_ok(cudaGetLastError());
 }
