@@ -1,0 +1,74 @@
+"""Training-set parallelism (Section 4.3) on two CPU ranks over gloo: each rank evaluates its slice of the seeded
+pattern stream with the CPU checker, the gradients are summed through the package's exchange, and every rank must
+end up with the gradient of the whole batch."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import oracle
+import synth_inputs as si
+from paper_1911_05181_b200 import dp
+
+SIZES = [12, 9, 5]
+PER_RANK = 37
+SEED = 31
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        Ws, bs = si.mlp_params(SEED, SIZES)
+        first, last = dp.shard_range(rank, world, PER_RANK)
+        X, y = si.mlp_batch(SEED, SIZES, last - first, offset=first)
+        loss, dW, db = oracle.mlp_gradient(Ws, bs, X, y)
+        grads = [torch.from_numpy(np.ascontiguousarray(g)) for g in dW + db]       # float64 on the CPU
+        loss_t = torch.tensor([loss], dtype=torch.float64)
+        ex = dp.GradientExchange(grads, dist)
+        ex.all_reduce(grads, loss_t)
+        np.savez(os.path.join(out_dir, "rank%d.npz" % rank), loss=loss_t.numpy(), *[g.numpy() for g in grads])
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_sum_to_the_full_batch(tmp_path):
+    world = 2
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    Ws, bs = si.mlp_params(SEED, SIZES)
+    X, y = si.mlp_batch(SEED, SIZES, world * PER_RANK)
+    loss, dW, db = oracle.mlp_gradient(Ws, bs, X, y)
+    for rank in range(world):
+        got = np.load(os.path.join(str(tmp_path), "rank%d.npz" % rank))
+        assert abs(got["loss"][0] - loss) <= 1e-12 * abs(loss)
+        for i, ref in enumerate(dW + db):
+            assert np.allclose(got["arr_%d" % i], ref, rtol=1e-12, atol=1e-14)
+
+
+def test_shard_arithmetic():
+    assert dp.shard_range(0, 4, 10) == (0, 10) and dp.shard_range(3, 4, 10) == (30, 40)
+    cover = [dp.split_range(163480, 8, r) for r in range(8)]             # a pattern count of Section 6.3
+    assert cover[0][0] == 0 and cover[-1][1] == 163480
+    assert all(a[1] == b[0] for a, b in zip(cover, cover[1:]))
+    assert max(b - a for a, b in cover) - min(b - a for a, b in cover) <= 1
+    with pytest.raises(ValueError):
+        dp.shard_range(4, 4, 10)
+
+
+def test_single_rank_exchange_is_a_no_op():
+    g = [torch.arange(6, dtype=torch.float32).reshape(2, 3), torch.ones(4)]
+    before = [t.clone() for t in g]
+    loss = torch.tensor([2.5], dtype=torch.float64)
+    dp.GradientExchange(g, None).all_reduce(g, loss)
+    assert all(torch.equal(a, b) for a, b in zip(g, before)) and loss.item() == 2.5
