@@ -293,6 +293,9 @@ struct ulsnn_mlp {
     int64_t stats_ld;
     // workspace carve-up
     float* H[MAX_LAYERS + 1];
+    float* Hlo[MAX_LAYERS + 1];     // 3xTF32: H_l is kept as a pair, H = tf32_rn(h) and Hlo the rounded remainder
+    float* Whi[MAX_LAYERS];         // 3xTF32: the same pair for every weight matrix, rebuilt at the start of a call
+    float* Wlo[MAX_LAYERS];
     float* D[MAX_LAYERS + 1];
     float* Z;
     float2* stats;
@@ -342,7 +345,13 @@ ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
         h->ldh[l] = round_up((int64_t)h->sizes[l] + 1, 4);
         h->ldd[l] = round_up((int64_t)h->sizes[l], 4);
         h->H[l] = (float*)take((size_t)B * h->ldh[l] * sizeof(float));
+        h->Hlo[l] = (h->math == ULSNN_MATH_3XTF32) ? (float*)take((size_t)B * h->ldh[l] * sizeof(float)) : nullptr;
         h->D[l] = (float*)take((size_t)B * h->ldd[l] * sizeof(float));
+    }
+    for (int l = 0; l < L; ++l) {
+        const size_t wbytes = (size_t)h->sizes[l] * h->sizes[l + 1] * sizeof(float);
+        h->Whi[l] = (h->math == ULSNN_MATH_3XTF32) ? (float*)take(wbytes) : nullptr;
+        h->Wlo[l] = (h->math == ULSNN_MATH_3XTF32) ? (float*)take(wbytes) : nullptr;
     }
     h->ldz = round_up((int64_t)h->sizes[L], 4);
     h->Z = (float*)take((size_t)B * h->ldz * sizeof(float));
@@ -377,6 +386,17 @@ void fill_handle(ulsnn_mlp* h, const ulsnn_mlp_desc_t* d) {
     for (int l = 0; l <= h->L; ++l) h->sizes[l] = d->sizes[l];
 }
 
+// B operand = weight matrix w (strides already set): the stored (hi, lo) pair where the tensor-core engine can take
+// it, the caller's matrix otherwise (the FFMA engine multiplies exact fp32 values anyway)
+void set_weight_operand(ulsnn_mlp* h, GemmDesc& d, const float* const* W, int w) {
+    d.B = W[w]; d.B_lo = nullptr;
+    if (h->math == ULSNN_MATH_3XTF32) {
+        GemmDesc t = d;
+        t.B = h->Whi[w]; t.B_lo = h->Wlo[w];
+        if (tc_gemm_supported(t)) d = t;
+    }
+}
+
 // run_gemm bracketed by events when the handle's timing is on
 ulsnn_status_t timed_gemm(ulsnn_mlp* h, const GemmDesc& d, cudaStream_t stream) {
     if (!h->timing || h->n_phases >= 3 * MAX_LAYERS) return run_gemm(d, h->math, stream);
@@ -397,23 +417,34 @@ ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* 
     const int L = h->L;
     h->n_phases = 0;
     if (h->timing) h->timed_calls++;
-    const float* in = X; int64_t ld_in = ldx;
+    // 3xTF32: every weight matrix is split once per call into its TF32 (hi, lo) pair, and the activations are
+    // written as such pairs, so that the products which read them need no operand pass for them
+    const bool pairs = h->math == ULSNN_MATH_3XTF32;
+    if (pairs) {
+        for (int l = 0; l < L; ++l) {
+            ulsnn_status_t st = launch_split_hilo(W[l], (int64_t)h->sizes[l] * h->sizes[l + 1], h->Whi[l], h->Wlo[l], stream);
+            if (st != ULSNN_OK) return st;
+        }
+    }
+    const float* in = X; const float* in_lo = nullptr; int64_t ld_in = ldx;
     for (int l = 1; l < L; ++l) {
         GemmDesc d{};
         d.M = n; d.N = h->sizes[l]; d.K = h->sizes[l - 1];
-        d.A = in; d.a_sm = ld_in; d.a_sk = 1;
-        d.B = W[l - 1]; d.b_sk = 1; d.b_sn = d.K;
-        d.C = h->H[l]; d.ldc = h->ldh[l]; d.alpha = 1.f; d.beta = 0.f;
+        d.A = in; d.A_lo = in_lo; d.a_sm = ld_in; d.a_sk = 1;
+        d.b_sk = 1; d.b_sn = d.K;
+        set_weight_operand(h, d, W, l - 1);
+        d.C = h->H[l]; d.C_lo = pairs ? h->Hlo[l] : nullptr; d.ldc = h->ldh[l]; d.alpha = 1.f; d.beta = 0.f;
         d.epi = EPI_BIAS_TANH; d.bias = b[l - 1]; d.ones_cols = (int)(h->ldh[l] - d.N);
         d.splits = 1; d.k_per_split = d.K;
         ulsnn_status_t st = timed_gemm(h, d, stream);
         if (st != ULSNN_OK) return st;
-        in = h->H[l]; ld_in = h->ldh[l];
+        in = h->H[l]; in_lo = d.C_lo; ld_in = h->ldh[l];
     }
     GemmDesc d{};
     d.M = n; d.N = h->sizes[L]; d.K = h->sizes[L - 1];
-    d.A = in; d.a_sm = ld_in; d.a_sk = 1;
-    d.B = W[L - 1]; d.b_sk = 1; d.b_sn = d.K;
+    d.A = in; d.A_lo = in_lo; d.a_sm = ld_in; d.a_sk = 1;
+    d.b_sk = 1; d.b_sn = d.K;
+    set_weight_operand(h, d, W, L - 1);
     d.C = keep_logits ? h->Z : nullptr; d.ldc = h->ldz; d.alpha = 1.f; d.beta = 0.f;
     d.epi = EPI_LOGITS; d.bias = b[L - 1]; d.labels = labels;
     d.stats = h->stats; d.stats_ld = h->stats_ld; d.zlabel = h->zlabel;
@@ -547,9 +578,10 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
         if (l + 1 == L) { d.A = h->Z; d.a_sm = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 1; }
         else            { d.A = h->D[l + 1]; d.a_sm = h->ldd[l + 1]; }
         d.a_sk = 1;
-        d.B = W[l]; d.b_sk = d.N; d.b_sn = 1;
+        d.b_sk = d.N; d.b_sn = 1;
+        set_weight_operand(h, d, W, l);
         d.C = h->D[l]; d.ldc = h->ldd[l]; d.alpha = 1.f; d.beta = 0.f;
-        d.epi = EPI_TANHP; d.Hm = h->H[l]; d.ldh = h->ldh[l];
+        d.epi = EPI_TANHP; d.Hm = h->H[l]; d.Hm_lo = h->Hlo[l]; d.ldh = h->ldh[l];
         d.colsum_part = (l == 1) ? h->colsum_parts : nullptr;
         d.splits = 1; d.k_per_split = d.K;
         if (l == 1) colsum_rows = ((n + 127) / 128) * (use_tc(d, h->math) ? tc_colsum_groups() : simt_colsum_groups());
@@ -565,7 +597,7 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
         if (w + 1 == L) { d.A = h->Z; d.a_sk = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 0; }
         else            { d.A = h->D[w + 1]; d.a_sk = h->ldd[w + 1]; }
         d.a_sm = 1;
-        if (w >= 1) { d.B = h->H[w]; d.b_sk = h->ldh[w]; } else { d.B = X; d.b_sk = ldx; }
+        if (w >= 1) { d.B = h->H[w]; d.B_lo = h->Hlo[w]; d.b_sk = h->ldh[w]; } else { d.B = X; d.b_sk = ldx; }
         d.b_sn = 1;
         d.alpha = 1.f; d.beta = 0.f; d.epi = EPI_PARTIAL;
         const bool tc = use_tc(d, h->math);

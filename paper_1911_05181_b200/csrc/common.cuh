@@ -21,13 +21,19 @@ struct GemmDesc {
     int64_t M, N, K;
     const float* A; int64_t a_sm, a_sk;   // A(i,k) = A[i*a_sm + k*a_sk]  (one of the strides is 1)
     const float* B; int64_t b_sk, b_sn;   // B(k,j) = B[k*b_sk + j*b_sn]
+    // Operands stored as a pair: when A_lo (B_lo) is not null the operand's value is A + A_lo, where A holds the
+    // values rounded to TF32 and A_lo the rounded remainders, with the strides of A (B).  The tensor-core engine
+    // then needs no operand pass for it in 3xTF32 mode; the FFMA engine adds the two.
+    const float* A_lo; const float* B_lo;
     float* C; int64_t ldc;
+    float* C_lo;              // BIAS_TANH: not null -> C gets tf32_rn(h) and C_lo the rounded remainder (same ldc)
     float alpha, beta;
     int epi;
     // epilogue operands
     const float* bias;        // [N]                 BIAS_TANH, LOGITS
     int ones_cols;            // BIAS_TANH: write C[:, N] = 1 and C[:, N+1 .. N+ones_cols) = 0 (0: nothing)
     const float* Hm; int64_t ldh;        // TANHP
+    const float* Hm_lo;       // TANHP: not null -> h = Hm + Hm_lo
     float* colsum_part;       // TANHP: [row_tiles * groups][N] partial column sums (may be null)
     const int32_t* labels;    // LOGITS and the A transform: label of each pattern
     float2* stats; int64_t stats_ld;     // LOGITS: stats[row*stats_ld + col_tile] = (max, sum exp(z - max))
@@ -82,6 +88,8 @@ ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* lse
                                    int64_t n, int64_t n_classes, float* parts, int accumulate, float* out,
                                    cudaStream_t stream);
 int delta_colsum_tiles(int64_t n);
+// hi[i] = tf32_rn(x[i]), lo[i] = tf32_rn(x[i] - hi[i])   (round to nearest, ties away from zero, 10 mantissa bits)
+ulsnn_status_t launch_split_hilo(const float* x, int64_t n, float* hi, float* lo, cudaStream_t stream);
 ulsnn_status_t launch_sgd(float* w, const float* g, int64_t n, float lr, cudaStream_t stream);
 ulsnn_status_t launch_zero(float* p, int64_t n, cudaStream_t stream);
 ulsnn_status_t launch_zero_f64(double* p, int64_t n, cudaStream_t stream);

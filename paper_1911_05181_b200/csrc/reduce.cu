@@ -100,6 +100,18 @@ __global__ void delta_colsum_kernel(const float* __restrict__ Z, int64_t ldz, co
     parts[(int64_t)blockIdx.y * n_classes + j] = s;
 }
 
+__device__ __forceinline__ float round_tf32(float x) {
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
+}
+
+__global__ void split_hilo_kernel(const float* __restrict__ x, int64_t n, float* __restrict__ hi, float* __restrict__ lo) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const float v = x[i], h = round_tf32(v);
+        hi[i] = h;
+        lo[i] = round_tf32(v - h);
+    }
+}
+
 __global__ void sgd_kernel(float* __restrict__ w, const float* __restrict__ g, int64_t n, float lr) {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         w[i] = fmaf(-lr, g[i], w[i]);
@@ -201,6 +213,13 @@ ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* lse
         if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
     }
     return launch_colsum_reduce(parts, tiles, n_classes, accumulate, out, stream);
+}
+
+ulsnn_status_t launch_split_hilo(const float* x, int64_t n, float* hi, float* lo, cudaStream_t stream) {
+    if (n <= 0) return ULSNN_OK;
+    split_hilo_kernel<<<grid_for(n, 256), 256, 0, stream>>>(x, n, hi, lo);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
 }
 
 ulsnn_status_t launch_sgd(float* w, const float* g, int64_t n, float lr, cudaStream_t stream) {

@@ -19,6 +19,7 @@ template <bool TRANSFORM>
 __device__ __forceinline__ float load_a(const GemmDesc& d, int64_t i, int64_t k, int64_t kend) {
     if (i >= d.M || k >= kend) return 0.f;
     float z = __ldg(d.A + i * d.a_sm + k * d.a_sk);
+    if (d.A_lo) z += __ldg(d.A_lo + i * d.a_sm + k * d.a_sk);
     if (TRANSFORM) {
         const int64_t p = d.a_pattern_is_m ? i : k;
         const int64_t c = d.a_pattern_is_m ? k : i;
@@ -29,7 +30,9 @@ __device__ __forceinline__ float load_a(const GemmDesc& d, int64_t i, int64_t k,
 
 __device__ __forceinline__ float load_b(const GemmDesc& d, int64_t k, int64_t j, int64_t kend) {
     if (j >= d.N || k >= kend) return 0.f;
-    return __ldg(d.B + k * d.b_sk + j * d.b_sn);
+    float v = __ldg(d.B + k * d.b_sk + j * d.b_sn);
+    if (d.B_lo) v += __ldg(d.B_lo + k * d.b_sk + j * d.b_sn);
+    return v;
 }
 
 template <int EPI, bool TRANSFORM>
@@ -130,11 +133,21 @@ __global__ void __launch_bounds__(NT) simt_gemm_kernel(const GemmDesc d) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int64_t c = col_of(j);
-                if (c < d.N) d.C[r * d.ldc + c] = tanhf(acc[i][j] + __ldg(d.bias + c));
+                if (c < d.N) {
+                    const float h = tanhf(acc[i][j] + __ldg(d.bias + c));
+                    if (d.C_lo) {
+                        const float hi = __uint_as_float((__float_as_uint(h) + 0x1000u) & 0xFFFFE000u);
+                        d.C[r * d.ldc + c] = hi;
+                        d.C_lo[r * d.ldc + c] = __uint_as_float((__float_as_uint(h - hi) + 0x1000u) & 0xFFFFE000u);
+                    } else {
+                        d.C[r * d.ldc + c] = h;
+                    }
+                }
             }
             if (d.ones_cols > 0 && tx == 0 && blockIdx.y == gridDim.y - 1) {
                 d.C[r * d.ldc + d.N] = 1.f;
                 for (int c = 1; c < d.ones_cols; ++c) d.C[r * d.ldc + d.N + c] = 0.f;
+                if (d.C_lo) for (int c = 0; c < d.ones_cols; ++c) d.C_lo[r * d.ldc + d.N + c] = 0.f;
             }
         }
     } else if (EPI == EPI_LOGITS) {
@@ -183,7 +196,8 @@ __global__ void __launch_bounds__(NT) simt_gemm_kernel(const GemmDesc d) {
             for (int j = 0; j < 8; ++j) {
                 const int64_t c = col_of(j);
                 if (c >= d.N) continue;
-                const float h = __ldg(d.Hm + r * d.ldh + c);
+                float h = __ldg(d.Hm + r * d.ldh + c);
+                if (d.Hm_lo) h += __ldg(d.Hm_lo + r * d.ldh + c);
                 const float o = (1.f - h * h) * acc[i][j];
                 d.C[r * d.ldc + c] = o;
                 cs[j] += o;

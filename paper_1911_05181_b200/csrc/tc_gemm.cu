@@ -64,6 +64,8 @@ struct TcParams {
     int b_tile_bytes;       // bytes of one CTA's B tile: (bn / CG) * 128
     int stage_bytes;
     int three_x, a_mn, b_mn, split_pass;
+    int a_pre, b_pre;       // 3xTF32: the operand arrives as a stored (hi, lo) pair, no operand pass for it
+    int c_pair;             // BIAS_TANH: the output is written as a (hi, lo) pair
     int chunk_blocks;       // k-blocks accumulated on one TMEM accumulator before it is added into the tile total
     int fast_math;          // TF32 mode: approximate exp
     int c_tma;              // the output (C or the split-K partials) is written with TMA stores
@@ -348,7 +350,8 @@ __device__ __forceinline__ void split4(const float4 x, float4& hi, float4& lo) {
 template <int EPI, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_c, const TcParams p) {
+               const __grid_constant__ CUtensorMap map_a_lo, const __grid_constant__ CUtensorMap map_b_lo,
+               const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c_lo, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128B swizzle pattern repeats every 8 rows of 128 bytes
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -406,7 +409,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // a K-major B tile is one box of bn/CG rows (rows past the matrix arrive as zeros); an MN-major one is
             // a box per 32 columns, and only the boxes the products read are fetched
             const int b_boxes = b_cols >> 5;
-            const uint32_t tx_bytes = (uint32_t)(A_TILE_BYTES + (p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes));
+            const uint32_t b_bytes = (uint32_t)(p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes);
+            const uint32_t tx_bytes = (uint32_t)A_TILE_BYTES * (p.a_pre ? 2u : 1u) + b_bytes * (p.b_pre ? 2u : 1u);
             int k0 = (int)kbeg;
             for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
                 const int s = rp.stage;
@@ -430,6 +434,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                         for (int g = 0; g < BN_MAX / 32; ++g)
                             if (g < b_boxes) tma_load_2d(sb + g * (BK * 128), &map_b, n0 + 32 * g, k0, bar);
+                    }
+                    // operands stored as (hi, lo) pairs: the lo tiles land beside the hi tiles
+                    if (p.a_pre) {
+                        const uint32_t sal = sa + off_a_lo;
+                        if (!p.a_mn) {
+                            tma_load_2d(sal, &map_a_lo, k0, m0, bar);
+                        } else {
+#pragma unroll
+                            for (int g = 0; g < BM / 32; ++g) tma_load_2d(sal + g * (BK * 128), &map_a_lo, m0 + 32 * g, k0, bar);
+                        }
+                    }
+                    if (p.b_pre) {
+                        const uint32_t sbl = sa + off_b_lo;
+                        if (!p.b_mn) {
+                            tma_load_2d(sbl, &map_b_lo, k0, n0, bar);
+                        } else {
+#pragma unroll
+                            for (int g = 0; g < BN_MAX / 32; ++g)
+                                if (g < b_boxes) tma_load_2d(sbl + g * (BK * 128), &map_b_lo, n0 + 32 * g, k0, bar);
+                        }
                     }
                 }
                 __syncwarp();
@@ -532,7 +556,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
         const bool c_vec = ((((uintptr_t)d.C) & 15) == 0) && ((d.ldc & 3) == 0);
         const bool bias_vec = (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) && ((((uintptr_t)d.bias) & 15) == 0);
-        const bool h_vec = (EPI == EPI_TANHP) && ((((uintptr_t)d.Hm) & 15) == 0) && ((d.ldh & 3) == 0);
+        const bool h_vec = (EPI == EPI_TANHP) && ((((uintptr_t)d.Hm) & 15) == 0) && ((((uintptr_t)d.Hm_lo) & 15) == 0) && ((d.ldh & 3) == 0);
         uint32_t tile_i = 0, stg_i = 0;
         uint32_t reads[2] = {0, 0};             // how often each TMEM region has been waited for
         bool ok = true;
@@ -648,17 +672,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 } else if (EPI == EPI_TANHP) {
                     if (rv) {
                         const float* hp = d.Hm + r * d.ldh + c0;
+                        const float* hl = d.Hm_lo ? d.Hm_lo + r * d.ldh + c0 : nullptr;
                         if (h_vec && full) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 4) {
-                                const float4 h = __ldg(reinterpret_cast<const float4*>(hp + j));
+                                float4 h = __ldg(reinterpret_cast<const float4*>(hp + j));
+                                if (hl) { const float4 l = __ldg(reinterpret_cast<const float4*>(hl + j)); h.x += l.x; h.y += l.y; h.z += l.z; h.w += l.w; }
                                 v[j] *= (1.f - h.x * h.x); v[j + 1] *= (1.f - h.y * h.y);
                                 v[j + 2] *= (1.f - h.z * h.z); v[j + 3] *= (1.f - h.w * h.w);
                             }
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                if (j < nvalid) { const float h = __ldg(hp + j); v[j] = (1.f - h * h) * v[j]; } else v[j] = 0.f;
+                                if (j < nvalid) { const float h = __ldg(hp + j) + (hl ? __ldg(hl + j) : 0.f); v[j] = (1.f - h * h) * v[j]; } else v[j] = 0.f;
                             }
                         }
                     } else {
@@ -667,8 +693,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                 }
 
-                // ---- store the 32x32 block
-                if (do_store) {
+                // ---- store the 32x32 block (through a swizzled staging block and a TMA store, or directly)
+                auto store_block = [&](const float (&w)[32], const CUtensorMap* map, float* direct_base, int64_t ld) {
                     if (p.c_tma) {
                         uint8_t* blk = stg + (stg_i & 1) * EPI_STAGE_BYTES;
                         ++stg_i;
@@ -678,23 +704,35 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         float4* rowp = reinterpret_cast<float4*>(blk + lane * 128);
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
-                            rowp[j ^ (lane & 7)] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            rowp[j ^ (lane & 7)] = make_float4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
                         proxy_fence_async();
                         __syncwarp();
                         if (lane == 0 && r0w < d.M) {
-                            tma_store_3d(&map_c, smem_u32(blk), c0, r0w, EPI == EPI_PARTIAL ? sp : 0);
+                            tma_store_3d(map, smem_u32(blk), c0, r0w, EPI == EPI_PARTIAL ? sp : 0);
                             bulk_commit();
                         }
                     } else if (rv) {
-                        float* dst = (EPI == EPI_PARTIAL) ? d.partials + ((int64_t)sp * d.M + r) * d.ldp + c0
-                                                          : d.C + r * d.ldc + c0;
+                        float* dst = direct_base + r * ld + c0;
                         if ((EPI == EPI_PARTIAL || c_vec) && full) {
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
                         } else {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
+                            for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = w[j];
                         }
+                    }
+                };
+                if (do_store) {
+                    if (EPI == EPI_PARTIAL) {
+                        store_block(v, &map_c, d.partials + (int64_t)sp * d.M * d.ldp, d.ldp);
+                    } else if (EPI == EPI_BIAS_TANH && p.c_pair) {
+                        float lo[32];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) { const float h = to_tf32(v[j]); lo[j] = to_tf32(v[j] - h); v[j] = h; }
+                        store_block(v, &map_c, d.C, d.ldc);
+                        store_block(lo, &map_c_lo, d.C_lo, d.ldc);
+                    } else {
+                        store_block(v, &map_c, d.C, d.ldc);
                     }
                 }
                 if (EPI == EPI_TANHP && d.colsum_part) {
@@ -718,6 +756,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (EPI == EPI_BIAS_TANH && d.ones_cols > 0 && nt == p.tiles_n - 1 && rv) {
                 d.C[r * d.ldc + d.N] = 1.f;
                 for (int cc = 1; cc < d.ones_cols; ++cc) d.C[r * d.ldc + d.N + cc] = 0.f;
+                if (p.c_pair) for (int cc = 0; cc < d.ones_cols; ++cc) d.C_lo[r * d.ldc + d.N + cc] = 0.f;
             }
         }
         if (lane == 0) bulk_wait_all();         // every store of this warp has left shared memory and is complete
@@ -767,6 +806,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 auto pass = [&](auto fast_tag, auto three_tag) {
                     constexpr bool FAST = decltype(fast_tag)::value, THREE = decltype(three_tag)::value;
                     constexpr int NA = (BM * BK / 4) / NT;          // 16-byte pieces of the A tile per thread
+                    if (!p.a_pre) {
                     float4 x[NA];
 #pragma unroll
                     for (int i = 0; i < NA; ++i) x[i] = a_hi[st + NT * i];
@@ -802,7 +842,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             a_hi[st + NT * i] = x[i];       // only reached when A was transformed
                         }
                     }
-                    if constexpr (THREE) {
+                    }
+                    if (THREE && !p.b_pre) {
                         const int nvec = b_cols * 8;                 // 128 bytes per column of the tile
 #pragma unroll 4
                         for (int idx = st; idx < nvec; idx += NT) {
@@ -904,9 +945,10 @@ int* status_ptr() {
     return ptr;
 }
 
+struct Maps { CUtensorMap a, b, a_lo, b_lo, c, c_lo; };
+
 template <int EPI, int CG>
-ulsnn_status_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const TcParams& p, int smem_bytes, int grid,
-                      cudaStream_t stream) {
+ulsnn_status_t launch(const Maps& m, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(tc_gemm_kernel<EPI, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
@@ -923,15 +965,14 @@ ulsnn_status_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtens
     attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG>, ma, mb, mc, p);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG>, m.a, m.b, m.a_lo, m.b_lo, m.c, m.c_lo, p);
     count_launch(1);
     return cuda_ok(e == cudaSuccess ? cudaGetLastError() : e);
 }
 
 template <int EPI>
-ulsnn_status_t launch_cg(int cg, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const TcParams& p, int smem_bytes,
-                         int grid, cudaStream_t stream) {
-    return cg == 2 ? launch<EPI, 2>(ma, mb, mc, p, smem_bytes, grid, stream) : launch<EPI, 1>(ma, mb, mc, p, smem_bytes, grid, stream);
+ulsnn_status_t launch_cg(int cg, const Maps& m, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
+    return cg == 2 ? launch<EPI, 2>(m, p, smem_bytes, grid, stream) : launch<EPI, 1>(m, p, smem_bytes, grid, stream);
 }
 
 }  // namespace
@@ -963,6 +1004,8 @@ bool tc_gemm_supported(const GemmDesc& d) {
     if (!b_k && d.b_sn != 1) return false;
     if (!operand_ok(d.A, a_k ? d.a_sm : d.a_sk, 0)) return false;
     if (!operand_ok(d.B, b_k ? d.b_sn : d.b_sk, 0)) return false;
+    if (d.A_lo && (((uintptr_t)d.A_lo) & 15) != 0) return false;
+    if (d.B_lo && (((uintptr_t)d.B_lo) & 15) != 0) return false;
     // logits as the A operand: either [pattern x class] read K-major or its transpose read MN-major
     if (d.a_transform && (a_k != (d.a_pattern_is_m != 0))) return false;
     return true;
@@ -984,7 +1027,9 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     if (units > 0x7fffffff) return ULSNN_ERR_TOO_LARGE;
     p.units = (int)units;
     p.three_x = three_x ? 1 : 0;
-    p.split_pass = (three_x || d.a_transform) ? 1 : 0;
+    p.a_pre = (three_x && d.A_lo && !d.a_transform) ? 1 : 0;
+    p.b_pre = (three_x && d.B_lo) ? 1 : 0;
+    p.split_pass = (d.a_transform || (three_x && !(p.a_pre && p.b_pre))) ? 1 : 0;
     p.fast_math = three_x ? 0 : 1;
     p.chunk_blocks = three_x ? 8 : (1 << 30);       // 256 elements of K per accumulator in the accurate mode
     p.b_tile_bytes = (p.bn / cg) * 128;
@@ -1000,33 +1045,41 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.status = status_ptr();
     if (!p.status) return ULSNN_ERR_CUDA;
 
-    CUtensorMap ma, mb;
-    const bool oka = p.a_mn ? make_map(&ma, d.A, d.M, d.K, d.a_sk, 32, 32, true) : make_map(&ma, d.A, d.K, d.M, d.a_sm, 32, BM, false);
-    const bool okb = p.b_mn ? make_map(&mb, d.B, d.N, d.K, d.b_sk, 32, 32, true) : make_map(&mb, d.B, d.K, d.N, d.b_sn, 32, p.bn / cg, false);
-    if (!oka || !okb) return ULSNN_ERR_CUDA;
+    Maps m;
+    memset(&m, 0, sizeof(m));
+    auto map_of_a = [&](CUtensorMap* t, const float* base) {
+        return p.a_mn ? make_map(t, base, d.M, d.K, d.a_sk, 32, 32, true) : make_map(t, base, d.K, d.M, d.a_sm, 32, BM, false);
+    };
+    auto map_of_b = [&](CUtensorMap* t, const float* base) {
+        return p.b_mn ? make_map(t, base, d.N, d.K, d.b_sk, 32, 32, true) : make_map(t, base, d.K, d.N, d.b_sn, 32, p.bn / cg, false);
+    };
+    if (!map_of_a(&m.a, d.A) || !map_of_b(&m.b, d.B)) return ULSNN_ERR_CUDA;
+    if (p.a_pre && !map_of_a(&m.a_lo, d.A_lo)) return ULSNN_ERR_CUDA;
+    if (p.b_pre && !map_of_b(&m.b_lo, d.B_lo)) return ULSNN_ERR_CUDA;
+    p.c_pair = (d.epi == EPI_BIAS_TANH && d.C_lo) ? 1 : 0;
 
     // the output goes through TMA stores when its rows are 16-byte aligned; otherwise the epilogue stores directly
-    CUtensorMap mc;
-    memset(&mc, 0, sizeof(mc));
     if (d.epi == EPI_PARTIAL) {
-        p.c_tma = make_store_map(&mc, d.partials, d.N, d.M, d.ldp, splits) ? 1 : 0;
+        p.c_tma = make_store_map(&m.c, d.partials, d.N, d.M, d.ldp, splits) ? 1 : 0;
     } else if (d.C && (((uintptr_t)d.C) & 15) == 0 && (d.ldc & 3) == 0 && d.ldc >= 4) {
         // A TMA store clips a row at the next 16-byte boundary past the matrix edge, so a width that is not a multiple
         // of four spills up to three floats into the row's padding.  That padding is scratch in the library's own
         // logit and delta buffers; it belongs to the caller in C, and it is the ones column in an activation buffer.
         const bool pad_is_scratch = d.epi == EPI_LOGITS || d.epi == EPI_TANHP;
-        if ((d.N & 3) == 0 || pad_is_scratch) p.c_tma = make_store_map(&mc, d.C, d.N, d.M, d.ldc, 1) ? 1 : 0;
+        if ((d.N & 3) == 0 || pad_is_scratch) p.c_tma = make_store_map(&m.c, d.C, d.N, d.M, d.ldc, 1) ? 1 : 0;
+        if (p.c_tma && p.c_pair)
+            p.c_tma = ((((uintptr_t)d.C_lo) & 15) == 0 && make_store_map(&m.c_lo, d.C_lo, d.N, d.M, d.ldc, 1)) ? 1 : 0;
     }
 
     const int smem_bytes = 1024 + stages * p.stage_bytes + EPI_SCRATCH_BYTES + CTRL_BYTES;
     const int slots = sm_count() / cg;
     const int grid = cg * (p.units < slots ? p.units : slots);
     switch (d.epi) {
-        case EPI_SGEMM:     return launch_cg<EPI_SGEMM>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
-        case EPI_BIAS_TANH: return launch_cg<EPI_BIAS_TANH>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
-        case EPI_LOGITS:    return launch_cg<EPI_LOGITS>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
-        case EPI_TANHP:     return launch_cg<EPI_TANHP>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
-        case EPI_PARTIAL:   return launch_cg<EPI_PARTIAL>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_SGEMM:     return launch_cg<EPI_SGEMM>(cg, m, p, smem_bytes, grid, stream);
+        case EPI_BIAS_TANH: return launch_cg<EPI_BIAS_TANH>(cg, m, p, smem_bytes, grid, stream);
+        case EPI_LOGITS:    return launch_cg<EPI_LOGITS>(cg, m, p, smem_bytes, grid, stream);
+        case EPI_TANHP:     return launch_cg<EPI_TANHP>(cg, m, p, smem_bytes, grid, stream);
+        case EPI_PARTIAL:   return launch_cg<EPI_PARTIAL>(cg, m, p, smem_bytes, grid, stream);
     }
     return ULSNN_ERR_INVALID_ARG;
 }
