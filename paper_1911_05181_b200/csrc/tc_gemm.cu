@@ -39,15 +39,17 @@ namespace {
 
 constexpr int BM = 128;                 // rows of an output tile (TMEM lanes)
 constexpr int BN_MAX = 256;             // widest column tile (TMEM columns per accumulator stage)
-constexpr int BK = 32;                  // fp32 elements per 128-byte swizzle row
+constexpr int BK = 32;                  // elements of K per pipeline stage (16 or 32): a K-major tile row is BK*4 bytes
+constexpr int ROW_BYTES = BK * 4;       // and is swizzled in 64-byte (BK = 16) or 128-byte (BK = 32) mode
+constexpr int CPR = ROW_BYTES / 16;     // 16-byte pieces per K-major row
 constexpr int UMMA_K = 8;               // K of one tcgen05.mma.kind::tf32
 constexpr int NUM_EPI_WARPS = 4;
 constexpr int NUM_SPLIT_WARPS = 8;
 constexpr int NUM_WARPS = 2 + NUM_EPI_WARPS + NUM_SPLIT_WARPS;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
-constexpr int MAX_STAGES = 8;
+constexpr int MAX_STAGES = 12;
 constexpr int NUM_SMS = 148;               // B200; fixes the tile schedule (and with it every summation order)
-constexpr int A_TILE_BYTES = BM * BK * 4;                       // 16 KB
+constexpr int A_TILE_BYTES = BM * BK * 4;
 constexpr int SMEM_BUDGET = 227 * 1024;
 constexpr int EPI_STAGE_BYTES = 32 * 128;                        // one 32x32 fp32 block, 128B-swizzled
 constexpr int EPI_SCRATCH_BYTES = NUM_EPI_WARPS * 2 * EPI_STAGE_BYTES;   // two store-staging blocks per epilogue warp
@@ -61,7 +63,7 @@ struct TcParams {
     int tiles_m, tiles_n;   // tiles_m counts tiles of 128*CG rows
     int units;              // tiles_m * tiles_n * splits
     int stages;
-    int b_tile_bytes;       // bytes of one CTA's B tile: (bn / CG) * 128
+    int b_tile_bytes;       // bytes of one CTA's B tile: (bn / CG) * BK * 4
     int stage_bytes;
     int three_x, a_mn, b_mn, split_pass;
     int a_pre, b_pre;       // 3xTF32: the operand arrives as a stored (hi, lo) pair, no operand pass for it
@@ -100,6 +102,18 @@ __device__ __forceinline__ void mbar_arrive_rank0(uint32_t bar) {
         "mapa.shared::cluster.u32 ra, %0, 0;\n\t"
         "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
         ::"r"(bar) : "memory");
+}
+// Asynchronous signal to CTA 0: stores 8 bytes into CTA 0's shared memory at the offset of `sink` and completes 8
+// transaction bytes on CTA 0's barrier at the offset of `bar`.  Unlike an arrival on a remote barrier it does not
+// hold up the sending thread.
+__device__ __forceinline__ void signal_rank0(uint32_t sink, uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .b32 rs, rb;\n\t.reg .b64 v;\n\t"
+        "mapa.shared::cluster.u32 rs, %0, 0;\n\t"
+        "mapa.shared::cluster.u32 rb, %1, 0;\n\t"
+        "mov.b64 v, 0;\n\t"
+        "st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b64 [rs], v, [rb];\n\t}"
+        ::"r"(sink), "r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -238,6 +252,7 @@ struct Ctrl {
     uint64_t empty[MAX_STAGES];     // products that read the stage have completed
     uint64_t reg_full[2];           // the products chained on TMEM region r have completed
     uint64_t reg_free[2];           // the epilogue warps have read region r: it may be overwritten
+    uint64_t relay_sink[MAX_STAGES];    // CTA 0: landing words of CTA 1's stage-ready signals
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -286,7 +301,7 @@ __device__ __forceinline__ void unit_k_range(const TcParams& p, int sp, int64_t&
     if (kend > p.d.K) kend = p.d.K;
     const int64_t len = kend - kbeg;
     nkb = (int)((len + BK - 1) / BK);
-    const int rem = (int)(len - (int64_t)(nkb - 1) * BK);      // 1..32 elements in the last block
+    const int rem = (int)(len - (int64_t)(nkb - 1) * BK);      // 1..BK elements in the last block
     tail_steps = (rem + UMMA_K - 1) / UMMA_K;
 }
 
@@ -362,9 +377,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const GemmDesc& d = p.d;
     // With CG == 2 the two CTAs of a cluster work on the same sequence of tiles.  CTA 0 issues the products.  Its
-    // `ready` barriers collect its own operand-pass warps and one arrival per stage that warp 1 of CTA 1 sends over
-    // when CTA 1's stage is ready (an arrival on another CTA's barrier costs its sender about a microsecond, so it
-    // is kept off the warps that do the work); its `reg_free` barriers collect the epilogue warps of both CTAs.
+    // `ready` barriers collect its own operand-pass warps and, per stage, 8 transaction bytes that warp 1 of CTA 1
+    // sends over with an asynchronous store when CTA 1's stage is ready (an arrival on another CTA's barrier holds
+    // its sender up for about a microsecond); its `reg_free` barriers collect the epilogue warps of both CTAs.
     const int rank = (CG == 2) ? (int)cluster_ctarank() : 0;
     const int first_unit = blockIdx.x / CG, unit_step = gridDim.x / CG;
 
@@ -422,14 +437,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (elect_one()) {
                     mbar_expect_tx(bar, tx_bytes);
                     if (!p.a_mn) {
-                        tma_load_2d(sa, &map_a, k0, m0, bar);                       // box {32 k, 128 rows}
+                        tma_load_2d(sa, &map_a, k0, m0, bar);                       // box {BK k, 128 rows}
                     } else {
 #pragma unroll
-                        for (int g = 0; g < BM / 32; ++g)                           // boxes {32 m, 32 k}
+                        for (int g = 0; g < BM / 32; ++g)                           // boxes {32 m, BK k}
                             tma_load_2d(sa + g * (BK * 128), &map_a, m0 + 32 * g, k0, bar);
                     }
                     if (!p.b_mn) {
-                        tma_load_2d(sb, &map_b, k0, n0, bar);                       // box {32 k, bn/CG rows}
+                        tma_load_2d(sb, &map_b, k0, n0, bar);                       // box {BK k, bn/CG rows}
                     } else {
 #pragma unroll
                         for (int g = 0; g < BN_MAX / 32; ++g)
@@ -464,12 +479,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (rank == 0) {
             const uint32_t idesc0 = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
                                     ((uint32_t)((BM * CG) >> 4) << 24);
-            // K-major (128B swizzle): 8-row groups 1024 B apart (SBO), K advance = 32 B inside the swizzled row.
+            // K-major (rows of BK*4 bytes, swizzled): 8-row groups 8*BK*4 B apart (SBO), K advance = 32 B inside the row.
             // MN-major (128B swizzle, 32-byte atoms): 32-element groups BK*128 B apart (LBO), 4-k groups 512 B apart
             // (SBO), K advance = 8 rows = 1024 B.
             const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
-            const uint32_t a_sbo = p.a_mn ? 512 : 1024, b_sbo = p.b_mn ? 512 : 1024;
-            const uint32_t a_lay = p.a_mn ? 1 : 2, b_lay = p.b_mn ? 1 : 2;
+            constexpr uint32_t K_SBO = 8 * ROW_BYTES, K_LAY = (BK == 32) ? 2 : 4;      // 8-row groups; 128B or 64B swizzle
+            const uint32_t a_sbo = p.a_mn ? 512 : K_SBO, b_sbo = p.b_mn ? 512 : K_SBO;
+            const uint32_t a_lay = p.a_mn ? 1 : K_LAY, b_lay = p.b_mn ? 1 : K_LAY;
             const uint32_t a_kstep = p.a_mn ? 1024 : UMMA_K * 4, b_kstep = p.b_mn ? 1024 : UMMA_K * 4;
             // descriptors of the four tiles of stage 0; a stage or a k step only moves the 14-bit start address
             const uint32_t base0 = smem_u32(stage_base);
@@ -501,6 +517,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                     const int s = rp.stage;
                     if (!p.split_pass && !wait_bar_warp(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
+                    // CTA 1's signal for this stage completes 8 transaction bytes on `ready`; posting the expectation is
+                    // this warp's own arrival on it
+                    if (CG == 2 && elect_one()) mbar_expect_tx(smem_u32(&ctrl->ready[s]), 8);
                     if ((p.split_pass || CG == 2) && !wait_bar_warp(&ctrl->ready[s], rp.phase, ctrl, p.status)) { ok = false; break; }
                     rp.advance(p.stages);
                     tc_fence_after();
@@ -543,7 +562,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     uint64_t* bar = p.split_pass ? &ctrl->ready[s] : &ctrl->full[s];
                     if (!wait_bar_warp(bar, rp.phase, ctrl, p.status)) { ok = false; break; }
                     rp.advance(p.stages);
-                    if (lane == 0) mbar_arrive_rank0(smem_u32(&ctrl->ready[s]));
+                    if (lane == 0) signal_rank0(smem_u32(&ctrl->relay_sink[s]), smem_u32(&ctrl->ready[s]));
                     __syncwarp();
                 }
             }
@@ -767,9 +786,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // Position of this thread's 16-byte pieces in the A tile (piece index st + 256*i, i = 0..3).
         //  K-major: row (st>>3) + 32*i of the tile, the four floats run along K from k0 + 4*kch
         //  MN-major: k row st>>3, the four floats run along M from m0 + 32*i + 4*mch
-        const int a_row = st >> 3;
-        const int kch = (st & 7) ^ (a_row & 7);
-        const int mch = ((((st & 7) >> 1) ^ (a_row & 3)) << 1) | (st & 1);
+        // K-major tile: piece idx = st + NT*i sits in row idx / CPR at position idx % CPR, which holds logical piece
+        // position ^ (row & 7) (128-byte rows) or position ^ ((row >> 1) & 3) (64-byte rows)
+        constexpr int ROW_STEP = NT / CPR;                      // rows between a thread's consecutive pieces
+        const int a_row = st / CPR;
+        const int kch = (st % CPR) ^ (BK == 32 ? (a_row & 7) : ((a_row >> 1) & 3));
+        // MN-major tile: 32-column groups of BK k rows of 128 bytes; piece idx sits in group idx / (BK*8), k row
+        // (idx % (BK*8)) / 8; 32-byte units of a row are XORed with (k row & 3)
+        constexpr int G_PIECES = BK * 8;                        // pieces per 32-column group
+        const int mn_g0 = st / G_PIECES, mn_gstep = NT / G_PIECES;          // group of piece i: mn_g0 + mn_gstep*i
+        const int mn_krow = (st % G_PIECES) >> 3;
+        const int mch = ((((st & 7) >> 1) ^ (mn_krow & 3)) << 1) | (st & 1);
         const int n_classes = (int)p.n_classes, n_patterns = (int)p.n_patterns;
         RingPos rp{0, 0};
         bool ok = true;
@@ -778,13 +805,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
             const int m0 = (mt * CG + rank) * BM;
             const int b_cols = tile_cols(p, nt) / CG;
-            // K-major logits (the pattern is the row): statistics of this thread's four rows, once per tile
-            float row_lse[4] = {0.f, 0.f, 0.f, 0.f};
-            int row_lab[4] = {-1, -1, -1, -1};
+            // K-major logits (the pattern is the row): statistics of this thread's rows, once per tile
+            constexpr int NA = (BM * BK / 4) / NT;          // 16-byte pieces of the A tile per thread
+            float row_lse[NA];
+            int row_lab[NA];
+#pragma unroll
+            for (int i = 0; i < NA; ++i) { row_lse[i] = 0.f; row_lab[i] = -1; }
             if (d.a_transform && !p.a_mn) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int pat = m0 + a_row + 32 * i;
+                for (int i = 0; i < NA; ++i) {
+                    const int pat = m0 + a_row + ROW_STEP * i;
                     if (pat < n_patterns) { row_lse[i] = __ldg(d.lse + pat); row_lab[i] = __ldg(d.labels + pat); }
                 }
             }
@@ -793,7 +823,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const int s = rp.stage;
                 // MN-major logits (the pattern is the k row): statistics of this thread's pattern in this block
                 float k_lse = 0.f; int k_lab = -1;
-                const int kpat = k0 + a_row;
+                const int kpat = k0 + mn_krow;
                 if (d.a_transform && p.a_mn && kpat < n_patterns) { k_lse = __ldg(d.lse + kpat); k_lab = __ldg(d.labels + kpat); }
                 if (!wait_bar(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
                 rp.advance(p.stages);
@@ -805,7 +835,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 // The body is instantiated per (approximate exp?, 3xTF32?) so that its unrolled loops are straight-line code.
                 auto pass = [&](auto fast_tag, auto three_tag) {
                     constexpr bool FAST = decltype(fast_tag)::value, THREE = decltype(three_tag)::value;
-                    constexpr int NA = (BM * BK / 4) / NT;          // 16-byte pieces of the A tile per thread
                     if (!p.a_pre) {
                     float4 x[NA];
 #pragma unroll
@@ -815,7 +844,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             const int cls = k0 + kch * 4;
 #pragma unroll
                             for (int i = 0; i < NA; ++i) {
-                                const bool live = m0 + a_row + 32 * i < n_patterns;
+                                const bool live = m0 + a_row + ROW_STEP * i < n_patterns;
                                 x[i].x = live ? delta_of<FAST>(x[i].x, row_lse[i], cls + 0, row_lab[i], n_classes) : 0.f;
                                 x[i].y = live ? delta_of<FAST>(x[i].y, row_lse[i], cls + 1, row_lab[i], n_classes) : 0.f;
                                 x[i].z = live ? delta_of<FAST>(x[i].z, row_lse[i], cls + 2, row_lab[i], n_classes) : 0.f;
@@ -825,7 +854,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             const bool live = kpat < n_patterns;
 #pragma unroll
                             for (int i = 0; i < NA; ++i) {
-                                const int cls = m0 + 32 * i + mch * 4;
+                                const int cls = m0 + 32 * (mn_g0 + mn_gstep * i) + mch * 4;
                                 x[i].x = live ? delta_of<FAST>(x[i].x, k_lse, cls + 0, k_lab, n_classes) : 0.f;
                                 x[i].y = live ? delta_of<FAST>(x[i].y, k_lse, cls + 1, k_lab, n_classes) : 0.f;
                                 x[i].z = live ? delta_of<FAST>(x[i].z, k_lse, cls + 2, k_lab, n_classes) : 0.f;
@@ -844,7 +873,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                     }
                     if (THREE && !p.b_pre) {
-                        const int nvec = b_cols * 8;                 // 128 bytes per column of the tile
+                        const int nvec = b_cols * CPR;               // BK*4 bytes per column of the tile
 #pragma unroll 4
                         for (int idx = st; idx < nvec; idx += NT) {
                             float4 h, l; split4(b_hi[idx], h, l);
@@ -896,7 +925,7 @@ EncodeTiledFn encode_fn() {
 }
 
 // Tensor map of a matrix whose contiguous dimension has `inner` elements and whose other dimension has `outer`
-// rows `stride_elems` apart; box = {box_inner (32 floats = one swizzle row), box_outer}.
+// rows `stride_elems` apart; box = {box_inner, box_outer}.
 bool make_map(CUtensorMap* map, const float* base, int64_t inner, int64_t outer, int64_t stride_elems, int box_inner, int box_outer,
               bool atom32) {
     EncodeTiledFn fn = encode_fn();
@@ -906,7 +935,8 @@ bool make_map(CUtensorMap* map, const float* base, int64_t inner, int64_t outer,
     cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void*)base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : (BK == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B),
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1031,8 +1061,8 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.b_pre = (three_x && d.B_lo) ? 1 : 0;
     p.split_pass = (d.a_transform || (three_x && !(p.a_pre && p.b_pre))) ? 1 : 0;
     p.fast_math = three_x ? 0 : 1;
-    p.chunk_blocks = three_x ? 8 : (1 << 30);       // 256 elements of K per accumulator in the accurate mode
-    p.b_tile_bytes = (p.bn / cg) * 128;
+    p.chunk_blocks = three_x ? 256 / BK : (1 << 30);       // 256 elements of K per accumulator in the accurate mode
+    p.b_tile_bytes = (p.bn / cg) * ROW_BYTES;
     p.stage_bytes = (A_TILE_BYTES + p.b_tile_bytes) * (three_x ? 2 : 1);
     int stages = (SMEM_BUDGET - 1024 - EPI_SCRATCH_BYTES - CTRL_BYTES) / p.stage_bytes;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -1048,10 +1078,10 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     Maps m;
     memset(&m, 0, sizeof(m));
     auto map_of_a = [&](CUtensorMap* t, const float* base) {
-        return p.a_mn ? make_map(t, base, d.M, d.K, d.a_sk, 32, 32, true) : make_map(t, base, d.K, d.M, d.a_sm, 32, BM, false);
+        return p.a_mn ? make_map(t, base, d.M, d.K, d.a_sk, 32, BK, true) : make_map(t, base, d.K, d.M, d.a_sm, BK, BM, false);
     };
     auto map_of_b = [&](CUtensorMap* t, const float* base) {
-        return p.b_mn ? make_map(t, base, d.N, d.K, d.b_sk, 32, 32, true) : make_map(t, base, d.K, d.N, d.b_sn, 32, p.bn / cg, false);
+        return p.b_mn ? make_map(t, base, d.N, d.K, d.b_sk, 32, BK, true) : make_map(t, base, d.K, d.N, d.b_sn, BK, p.bn / cg, false);
     };
     if (!map_of_a(&m.a, d.A) || !map_of_b(&m.b, d.B)) return ULSNN_ERR_CUDA;
     if (p.a_pre && !map_of_a(&m.a_lo, d.A_lo)) return ULSNN_ERR_CUDA;
