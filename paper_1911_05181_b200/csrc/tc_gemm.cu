@@ -95,14 +95,6 @@ __device__ __forceinline__ bool elect_one() {
     asm volatile("{\n\t.reg .pred px;\n\telect.sync _|px, 0xffffffff;\n\t@px mov.s32 %0, 1;\n\t}" : "+r"(pred));
     return pred != 0;
 }
-// arrive on the barrier at the same shared-memory offset in CTA 0 of the cluster (which may be this CTA)
-__device__ __forceinline__ void mbar_arrive_rank0(uint32_t bar) {
-    asm volatile(
-        "{\n\t.reg .b32 ra;\n\t"
-        "mapa.shared::cluster.u32 ra, %0, 0;\n\t"
-        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
-        ::"r"(bar) : "memory");
-}
 // Asynchronous signal to CTA 0: stores 8 bytes into CTA 0's shared memory at the offset of `sink` and completes 8
 // transaction bytes on CTA 0's barrier at the offset of `bar`.  Unlike an arrival on a remote barrier it does not
 // hold up the sending thread.
@@ -253,6 +245,7 @@ struct Ctrl {
     uint64_t reg_full[2];           // the products chained on TMEM region r have completed
     uint64_t reg_free[2];           // the epilogue warps have read region r: it may be overwritten
     uint64_t relay_sink[MAX_STAGES];    // CTA 0: landing words of CTA 1's stage-ready signals
+    uint64_t free_sink[2][NUM_EPI_WARPS];   // CTA 0: landing words of CTA 1's accumulator-free signals
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -379,7 +372,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // With CG == 2 the two CTAs of a cluster work on the same sequence of tiles.  CTA 0 issues the products.  Its
     // `ready` barriers collect its own operand-pass warps and, per stage, 8 transaction bytes that warp 1 of CTA 1
     // sends over with an asynchronous store when CTA 1's stage is ready (an arrival on another CTA's barrier holds
-    // its sender up for about a microsecond); its `reg_free` barriers collect the epilogue warps of both CTAs.
+    // its sender up for about a microsecond); its `reg_free` barriers collect its own epilogue warps and 8 bytes
+    // from each epilogue warp of CTA 1 in the same way.
     const int rank = (CG == 2) ? (int)cluster_ctarank() : 0;
     const int first_unit = blockIdx.x / CG, unit_step = gridDim.x / CG;
 
@@ -393,7 +387,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&ctrl->reg_full[a]), 1);
-            mbar_init(smem_u32(&ctrl->reg_free[a]), CG * NUM_EPI_WARPS);
+            // CTA 0: its epilogue warps, plus (CG == 2) the issuing warp's own arrival that posts the 8 bytes each of
+            // CTA 1's epilogue warps will signal
+            mbar_init(smem_u32(&ctrl->reg_free[a]), NUM_EPI_WARPS + (CG == 2 ? 1 : 0));
         }
         ctrl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -510,7 +506,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (chunk_start) {
                         // chunk 0 goes to the tile's total region, later chunks restart the other region
                         reg = (kb == 0) ? total_reg : (total_reg ^ 1);
-                        if (!wait_bar_warp(&ctrl->reg_free[reg], (overwrites[reg] & 1) ^ 1, ctrl, p.status)) { ok = false; break; }
+                        if (overwrites[reg] > 0) {          // the region has been used: wait until both CTAs have read it
+                            if (CG == 2 && elect_one()) mbar_expect_tx(smem_u32(&ctrl->reg_free[reg]), 8 * NUM_EPI_WARPS);
+                            if (!wait_bar_warp(&ctrl->reg_free[reg], (overwrites[reg] - 1) & 1, ctrl, p.status)) { ok = false; break; }
+                        }
                         overwrites[reg]++;
                         tc_fence_after();
                         d_tmem = tmem_base + reg * BN_MAX;
@@ -606,7 +605,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) { if constexpr (CG == 2) mbar_arrive_rank0(smem_u32(&ctrl->reg_free[oth])); else mbar_arrive(smem_u32(&ctrl->reg_free[oth])); }
+                if (lane == 0) { if (CG == 2 && rank == 1) signal_rank0(smem_u32(&ctrl->free_sink[oth][ew]), smem_u32(&ctrl->reg_free[oth])); else mbar_arrive(smem_u32(&ctrl->reg_free[oth])); }
             }
             if (!ok) break;
             const int r0w = (mt * CG + rank) * BM + q * 32;   // first row of this warp's 32-row block
@@ -766,7 +765,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // all TMEM reads of this accumulator stage are done: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) { if constexpr (CG == 2) mbar_arrive_rank0(smem_u32(&ctrl->reg_free[acc])); else mbar_arrive(smem_u32(&ctrl->reg_free[acc])); }
+            if (lane == 0) { if (CG == 2 && rank == 1) signal_rank0(smem_u32(&ctrl->free_sink[acc][ew]), smem_u32(&ctrl->reg_free[acc])); else mbar_arrive(smem_u32(&ctrl->reg_free[acc])); }
 
             if (EPI == EPI_LOGITS && rv) {
                 d.stats[r * d.stats_ld + nt] = make_float2(run_m, run_s);
