@@ -298,6 +298,7 @@ struct ulsnn_mlp {
     float* Wlo[MAX_LAYERS];
     float* D[MAX_LAYERS + 1];
     float* Z;
+    float* D2; float* D2lo;         // delta of the output layer as left behind by the first delta product (pair in 3xTF32)
     float2* stats;
     float* lse;
     float* zlabel;
@@ -355,6 +356,10 @@ ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
     }
     h->ldz = round_up((int64_t)h->sizes[L], 4);
     h->Z = (float*)take((size_t)B * h->ldz * sizeof(float));
+    // TF32 mode only: in 3xTF32 mode storing the (hi, lo) tiles slowed the delta product down by more than the
+    // weight-gradient product gained (measured 1.15 -> 1.57 ms against 1.18 -> 0.89 ms at 65536 patterns)
+    h->D2 = (L >= 2 && h->math == ULSNN_MATH_TF32) ? (float*)take((size_t)B * h->ldz * sizeof(float)) : nullptr;
+    h->D2lo = nullptr;
     h->stats_ld = ((int64_t)h->sizes[L] + 63) / 64;          // enough for any column-tile width >= 64
     h->stats = (float2*)take((size_t)B * h->stats_ld * sizeof(float2));
     h->lse = (float*)take((size_t)B * sizeof(float));
@@ -570,12 +575,16 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
     if ((st = forward(h, W, b, X, ldx, labels, n, true, accumulate, loss_out, stream)) != ULSNN_OK) return st;
 
     int64_t colsum_rows = 0;
+    bool delta2_kept = false;       // the top delta product ran on the tensor-core engine and left delta_L in D2
     // Deltas of the hidden layers, top down: delta_l = (1 - H_l*H_l) * (delta_{l+1} W_{l+1})   (H_D of Section 4.2).
     // delta_L is never stored: the kernels form softmax(z) - onehot from the logits as they load them.
     for (int l = L - 1; l >= 1; --l) {
         GemmDesc d{};
         d.M = n; d.N = h->sizes[l]; d.K = h->sizes[l + 1];
-        if (l + 1 == L) { d.A = h->Z; d.a_sm = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 1; }
+        if (l + 1 == L) {
+            d.A = h->Z; d.a_sm = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 1;
+            d.delta_out = h->D2; d.delta_out_lo = h->D2lo;      // kept for the weight-gradient product below
+        }
         else            { d.A = h->D[l + 1]; d.a_sm = h->ldd[l + 1]; }
         d.a_sk = 1;
         d.b_sk = d.N; d.b_sn = 1;
@@ -584,6 +593,7 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
         d.epi = EPI_TANHP; d.Hm = h->H[l]; d.Hm_lo = h->Hlo[l]; d.ldh = h->ldh[l];
         d.colsum_part = (l == 1) ? h->colsum_parts : nullptr;
         d.splits = 1; d.k_per_split = d.K;
+        if (l + 1 == L) delta2_kept = use_tc(d, h->math) && tc_keeps_delta(d, h->math == ULSNN_MATH_3XTF32);
         if (l == 1) colsum_rows = ((n + 127) / 128) * (use_tc(d, h->math) ? tc_colsum_groups() : simt_colsum_groups());
         if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
     }
@@ -594,7 +604,8 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
     for (int w = L - 1; w >= 0; --w) {
         GemmDesc d{};
         d.M = h->sizes[w + 1]; d.N = h->sizes[w] + (w >= 1 ? 1 : 0); d.K = n;
-        if (w + 1 == L) { d.A = h->Z; d.a_sk = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 0; }
+        if (w + 1 == L && delta2_kept) { d.A = h->D2; d.A_lo = h->D2lo; d.a_sk = h->ldz; }
+        else if (w + 1 == L) { d.A = h->Z; d.a_sk = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 0; }
         else            { d.A = h->D[w + 1]; d.a_sk = h->ldd[w + 1]; }
         d.a_sm = 1;
         if (w >= 1) { d.B = h->H[w]; d.B_lo = h->Hlo[w]; d.b_sk = h->ldh[w]; } else { d.B = X; d.b_sk = ldx; }

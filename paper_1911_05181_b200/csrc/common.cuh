@@ -42,6 +42,10 @@ struct GemmDesc {
     int a_transform;
     const float* lse;         // [patterns] log-sum-exp of each pattern's logits
     int a_pattern_is_m;       // 1: the M index of A is the pattern (K is the class); 0: K is the pattern
+    // Optional copy of the transformed operand (tensor-core engine, a_pattern_is_m == 1 only): delta = softmax - onehot
+    // is also written to delta_out (and, in 3xTF32 mode, as the pair tf32_rn(delta) -> delta_out, remainder ->
+    // delta_out_lo), [patterns x classes] with the row stride of A, for the product that needs it next.
+    float* delta_out; float* delta_out_lo;
     // split-K (EPI_PARTIAL): slice s covers k in [s*k_per_split, min(K, (s+1)*k_per_split))
     int splits; int64_t k_per_split;
     float* partials; int64_t ldp;        // partials[(s*M + i)*ldp + j]
@@ -57,6 +61,8 @@ int simt_tile_n();
 // tcgen05 engine (tc_gemm.cu).  tc_gemm_supported: can TMA address these operands (16-byte aligned bases, leading
 // dimensions that are multiples of 4 floats)?  tc_tile_n: the column-tile width it will use for this product.
 bool tc_gemm_supported(const GemmDesc& d);
+// will the tensor-core engine leave the transformed operand in d.delta_out (see GemmDesc)?
+bool tc_keeps_delta(const GemmDesc& d, bool three_x);
 int tc_tile_m(const GemmDesc& d);
 int tc_tile_n(const GemmDesc& d);
 // how many tiles each engine works on at a time (CTAs, or CTA pairs): what a split-K plan has to fill
