@@ -30,7 +30,11 @@ WORKLOADS = {
     "config1": ([256, 128, 64], 4096, 0),
     "config3": ([400, 480, 3203], 65536, 2),
     "config5": ([1024, 4096, 4096, 3203], 131072, 4),
+    # one step = one pass over 9,000,000 resident patterns in 131072-pattern chunks accumulated in a fixed order
+    # (Section 4.3), then the parameter step; use --steps 5 or so (a step takes about half a second)
+    "config4": ([400, 480, 3203], 9_000_000, 3),
 }
+CHUNK = {"config4": 131072}
 MATH = {"3xtf32": 0, "tf32": 1, "simt": 2}
 NOMINAL_TF32_OVER_BF16 = 0.5        # dense TF32 tensor rate is half the BF16 rate
 # DRAM bytes per launch of the dominant kernel from one ncu capture (profiles/tc_gemm_3xtf32_config3.md: measured at
@@ -210,13 +214,19 @@ def main():
     Xh = torch.empty(batch, sizes[0], pin_memory=True); yh = torch.empty(batch, dtype=torch.int32, pin_memory=True)
     Xh.copy_(X); yh.copy_(y)
     loss_h = torch.zeros(1, dtype=torch.float64, pin_memory=True)
-    net = ul.Mlp(sizes, math_mode, batch)
+    chunk = min(batch, CHUNK.get(args.workload, batch))
+    starts = list(range(0, batch, chunk))
+    net = ul.Mlp(sizes, math_mode, chunk)
     lr = 1e-3 / (batch * world)
     stream = torch.cuda.current_stream()
     exchange = dp.GradientExchange(dW + db, dist)
 
-    def step(Xd, yd):
-        net.gradient(W, b, Xd, sizes[0], yd, batch, False, dW, db, loss)
+    def step(Xd, yd, host=None):
+        for i, lo in enumerate(starts):
+            hi = min(batch, lo + chunk)
+            if host is not None:            # end-to-end leg: this chunk's patterns come from pinned host memory
+                Xd[lo:hi].copy_(host[0][lo:hi], non_blocking=True); yd[lo:hi].copy_(host[1][lo:hi], non_blocking=True)
+            net.gradient(W, b, Xd[lo:hi], sizes[0], yd[lo:hi], hi - lo, i > 0, dW, db, loss)
         # the one exchange step of the method: sum of the per-rank gradients and losses (Section 4.3), NCCL
         exchange.all_reduce(dW + db, loss)
         net.sgd_step(W, b, dW, db, lr)
@@ -264,8 +274,7 @@ def main():
     reset_params()
 
     def e2e_step():
-        X.copy_(Xh, non_blocking=True); y.copy_(yh, non_blocking=True)
-        step(X, y)
+        step(X, y, host=(Xh, yh))
         loss_h.copy_(loss, non_blocking=True)
 
     for _ in range(2):
@@ -313,7 +322,7 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline:
-        n_sample = {"config1": 4096, "config3": 16384, "config5": 1024}[args.workload]
+        n_sample = {"config1": 4096, "config3": 16384, "config5": 1024, "config4": 16384}[args.workload]
         cpu = cpu_baseline(sizes, seed, min(batch, n_sample))
 
     line = {
@@ -333,7 +342,7 @@ def main():
         "launch_kinds": {k: int(c1[k] - c0[k]) for k in c1},
         "roofline": roofline,
         "phases_ms": [{"ms": round(p[0], 4), "M": p[1], "N": p[2], "K": p[3]} for p in phases],
-        "gemm_share_of_step": gemm_ms / ms_step if ms_step else None,
+        "gemm_share_of_step": gemm_ms / ms_step if ms_step and len(starts) == 1 else None,
         "cpu_baseline": cpu,
         "clocks": clocks,
         "device_status": status,
