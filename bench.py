@@ -110,15 +110,19 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def cpu_baseline(sizes, seed, n_sample):
+def cpu_baseline(sizes, seed, n_sample, head="softmax"):
     """The CPU checker, as it stands, on the first n_sample patterns of the workload."""
     import oracle
     import synth_inputs as si
     from paper_1911_05181_b200 import flops
     Ws, bs = si.mlp_params(seed, sizes)
     X, y = si.mlp_batch(seed, sizes, n_sample)
+    T = si.mlp_targets(seed, sizes, n_sample) if head == "sse" else None
     t0 = time.perf_counter()
-    oracle.mlp_gradient(Ws, bs, X, y)
+    if head == "sse":
+        oracle.mlp_sse_gradient(Ws, bs, X, T)
+    else:
+        oracle.mlp_gradient(Ws, bs, X, y)
     dt = time.perf_counter() - t0
     return {"value": flops.gradient_flops(sizes, n_sample) / dt / 1e9, "unit": "GFLOP/s", "cores": oracle.num_threads(),
             "kind": "oracle", "sample": "first %d patterns of the batch, one gradient evaluation, %.1f s" % (n_sample, dt),
@@ -172,6 +176,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--math", default="3xtf32", choices=sorted(MATH))
     ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS))
+    ap.add_argument("--head", default="softmax", choices=["softmax", "sse"],
+                    help="softmax + cross-entropy on labels (the benchmark's workload) or the paper's tanh outputs with "
+                         "summed squared error on a dense target matrix")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--patterns", type=int, default=0,
                     help="patterns per GPU instead of the workload's own count (for profiler captures of a smaller case)")
@@ -211,7 +218,10 @@ def main():
     first, _ = dp.shard_range(rank, world, batch)
     ul.fill_uniform(X, X.numel(), seed, si.TID_X, first * sizes[0], 0)
     ul.fill_labels(y, batch, seed, si.TID_LABELS, first, sizes[-1])
-    Xh = torch.empty(batch, sizes[0], pin_memory=True); yh = torch.empty(batch, dtype=torch.int32, pin_memory=True)
+    if args.head == "sse":       # dense targets uniform [-1, 1) in place of the labels
+        y = torch.empty(batch, sizes[-1], device="cuda")
+        ul.fill_uniform(y, y.numel(), seed, si.TID_TARGETS, first * sizes[-1], 1)
+    Xh = torch.empty(batch, sizes[0], pin_memory=True); yh = torch.empty(y.shape, dtype=y.dtype, pin_memory=True)
     Xh.copy_(X); yh.copy_(y)
     loss_h = torch.zeros(1, dtype=torch.float64, pin_memory=True)
     chunk = min(batch, CHUNK.get(args.workload, batch))
@@ -226,7 +236,10 @@ def main():
             hi = min(batch, lo + chunk)
             if host is not None:            # end-to-end leg: this chunk's patterns come from pinned host memory
                 Xd[lo:hi].copy_(host[0][lo:hi], non_blocking=True); yd[lo:hi].copy_(host[1][lo:hi], non_blocking=True)
-            net.gradient(W, b, Xd[lo:hi], sizes[0], yd[lo:hi], hi - lo, i > 0, dW, db, loss)
+            if args.head == "sse":
+                net.gradient_sse(W, b, Xd[lo:hi], sizes[0], yd[lo:hi], sizes[-1], hi - lo, i > 0, dW, db, loss)
+            else:
+                net.gradient(W, b, Xd[lo:hi], sizes[0], yd[lo:hi], hi - lo, i > 0, dW, db, loss)
         # the one exchange step of the method: sum of the per-rank gradients and losses (Section 4.3), NCCL
         exchange.all_reduce(dW + db, loss)
         net.sgd_step(W, b, dW, db, lr)
@@ -323,14 +336,14 @@ def main():
     cpu = None
     if not args.no_cpu_baseline:
         n_sample = {"config1": 4096, "config3": 16384, "config5": 1024, "config4": 16384}[args.workload]
-        cpu = cpu_baseline(sizes, seed, min(batch, n_sample))
+        cpu = cpu_baseline(sizes, seed, min(batch, n_sample), args.head)
 
     line = {
         "metric": "gradient_eval_gflops", "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "%s: %s MLP, %d patterns per GPU, seed %d" % (args.workload, "-".join(map(str, sizes)), batch, seed),
-                   "math": args.math, "global_batch": batch * world, "parallelism": "dp%d" % world,
+                   "math": args.math, "head": args.head, "global_batch": batch * world, "parallelism": "dp%d" % world,
                    "l2": "no flush: inputs and intermediates of a step (X %.0f MB, logits %.0f MB) exceed the 126 MB L2"
                          % (batch * sizes[0] * 4 / 1e6, batch * sizes[-1] * 4 / 1e6),
                    "step": "gradient evaluation + W -= lr*grad, lr = 1e-3 / global_batch"},

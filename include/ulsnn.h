@@ -159,6 +159,22 @@ ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* handle, const float* const* W, co
                                   const float* X, int64_t ldx, const int32_t* labels, int64_t n_patterns,
                                   int accumulate, float* const* dW, float* const* db, double* loss_out,
                                   ulsnn_stream_t stream);
+/*
+ * The paper's own output layer and error (Section 4.1): tanh output units, Eq. 1, and the summed squared error of
+ * Eq. 3, E = sum_p sum_j (y_pj - t_pj)^2 with y = tanh(W_L h + b_L), against a dense target matrix.
+ * T is [n_patterns x sizes[L]] fp32 device memory, row-major, ldt >= sizes[L] (any values: +-1 codes, 0/1 codes ...).
+ * ulsnn_mlp_forward_sse writes E to *loss_out; ulsnn_mlp_gradient_sse also returns dE/dW[l] and dE/db[l], the true
+ * derivatives of Eq. 3: the matrices of Section 4.2 built from Y_D = (1 - Y*Y)*(T - Y) equal -1/2 times these.
+ * Everything else (hidden layers, accumulate, summation over patterns, n_patterns == 0, errors) is as in
+ * ulsnn_mlp_forward_loss / ulsnn_mlp_gradient; the flop count is the same (Section 6.2).
+ */
+ulsnn_status_t ulsnn_mlp_forward_sse(ulsnn_mlp_t* handle, const float* const* W, const float* const* b,
+                                     const float* X, int64_t ldx, const float* T, int64_t ldt, int64_t n_patterns,
+                                     double* loss_out, ulsnn_stream_t stream);
+ulsnn_status_t ulsnn_mlp_gradient_sse(ulsnn_mlp_t* handle, const float* const* W, const float* const* b,
+                                      const float* X, int64_t ldx, const float* T, int64_t ldt, int64_t n_patterns,
+                                      int accumulate, float* const* dW, float* const* db, double* loss_out,
+                                      ulsnn_stream_t stream);
 /* Section 4.2: W := W - lr * dW, b := b - lr * db, in place, one fused multiply-add per element. */
 ulsnn_status_t ulsnn_sgd_step(ulsnn_mlp_t* handle, float* const* W, float* const* b,
                               const float* const* dW, const float* const* db, float lr, ulsnn_stream_t stream);

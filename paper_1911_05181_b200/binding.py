@@ -30,7 +30,7 @@ EXPORTS = [
     "ulsnn_mlp_workspace_bytes", "ulsnn_mlp_create", "ulsnn_mlp_destroy", "ulsnn_mlp_forward_loss",
     "ulsnn_mlp_gradient", "ulsnn_sgd_step", "ulsnn_last_device_status", "ulsnn_fill_uniform",
     "ulsnn_fill_labels", "ulsnn_launch_counts", "ulsnn_mlp_enable_timing", "ulsnn_mlp_phase_times",
-    "ulsnn_sgemm_noalloc", "ulsnn_sgemm_noalloc_max_scratch_bytes",
+    "ulsnn_sgemm_noalloc", "ulsnn_sgemm_noalloc_max_scratch_bytes", "ulsnn_mlp_forward_sse", "ulsnn_mlp_gradient_sse",
 ]
 
 
@@ -74,6 +74,8 @@ def lib():
         pp = ctypes.POINTER(vp)
         l.ulsnn_mlp_forward_loss.argtypes = [vp, pp, pp, vp, i64, vp, i64, vp, vp]
         l.ulsnn_mlp_gradient.argtypes = [vp, pp, pp, vp, i64, vp, i64, ctypes.c_int, pp, pp, vp, vp]
+        l.ulsnn_mlp_forward_sse.argtypes = [vp, pp, pp, vp, i64, vp, i64, i64, vp, vp]
+        l.ulsnn_mlp_gradient_sse.argtypes = [vp, pp, pp, vp, i64, vp, i64, i64, ctypes.c_int, pp, pp, vp, vp]
         l.ulsnn_sgd_step.argtypes = [vp, pp, pp, pp, pp, f32, vp]
         l.ulsnn_last_device_status.argtypes = [vp, vp]
         l.ulsnn_fill_uniform.argtypes = [vp, i64, u64, u64, u64, ctypes.c_int, vp]
@@ -223,6 +225,21 @@ class Mlp:
                                       _stream(stream))
         if check:
             _check(st, "ulsnn_mlp_gradient")
+        return st
+
+    def forward_sse(self, W, b, X, ldx, T, ldt, n_patterns, loss_out, stream=None, check=True):
+        st = lib().ulsnn_mlp_forward_sse(self._h, _ptr_array(W), _ptr_array(b), _ptr(X), ldx, _ptr(T), ldt,
+                                         n_patterns, _ptr(loss_out), _stream(stream))
+        if check:
+            _check(st, "ulsnn_mlp_forward_sse")
+        return st
+
+    def gradient_sse(self, W, b, X, ldx, T, ldt, n_patterns, accumulate, dW, db, loss_out, stream=None, check=True):
+        st = lib().ulsnn_mlp_gradient_sse(self._h, _ptr_array(W), _ptr_array(b), _ptr(X), ldx, _ptr(T), ldt, n_patterns,
+                                          1 if accumulate else 0, _ptr_array(dW), _ptr_array(db), _ptr(loss_out),
+                                          _stream(stream))
+        if check:
+            _check(st, "ulsnn_mlp_gradient_sse")
         return st
 
     def sgd_step(self, W, b, dW, db, lr, stream=None, check=True):

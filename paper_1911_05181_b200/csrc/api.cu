@@ -299,6 +299,7 @@ struct ulsnn_mlp {
     float* D[MAX_LAYERS + 1];
     float* Z;
     float* D2; float* D2lo;         // delta of the output layer as left behind by the first delta product (pair in 3xTF32)
+    float* Zlo;                     // 3xTF32, squared-error head: lo half of the output deltas (Z holds the hi half)
     float2* stats;
     float* lse;
     float* zlabel;
@@ -360,6 +361,7 @@ ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
     // weight-gradient product gained (measured 1.15 -> 1.57 ms against 1.18 -> 0.89 ms at 65536 patterns)
     h->D2 = (L >= 2 && h->math == ULSNN_MATH_TF32) ? (float*)take((size_t)B * h->ldz * sizeof(float)) : nullptr;
     h->D2lo = nullptr;
+    h->Zlo = (h->math == ULSNN_MATH_3XTF32) ? (float*)take((size_t)B * h->ldz * sizeof(float)) : nullptr;
     h->stats_ld = ((int64_t)h->sizes[L] + 63) / 64;          // enough for any column-tile width >= 64
     h->stats = (float2*)take((size_t)B * h->stats_ld * sizeof(float2));
     h->lse = (float*)take((size_t)B * sizeof(float));
@@ -416,9 +418,14 @@ ulsnn_status_t timed_gemm(ulsnn_mlp* h, const GemmDesc& d, cudaStream_t stream) 
 }
 
 // The forward products: hidden layers with bias + tanh fused, then the logits with their row statistics.
+// What the outputs are compared with: integer labels (softmax + cross-entropy) or, when T is not null, a dense
+// target matrix (the paper's tanh outputs with summed squared error, Eqs. 1 and 3).
+struct Targets { const int32_t* labels; const float* T; int64_t ldt; };
+
 ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
-                       const int32_t* labels, int64_t n, bool keep_logits, int accumulate, double* loss_out,
+                       const Targets& tg, int64_t n, bool keep_logits, int accumulate, double* loss_out,
                        cudaStream_t stream) {
+    const int32_t* labels = tg.labels;
     const int L = h->L;
     h->n_phases = 0;
     if (h->timing) h->timed_calls++;
@@ -452,6 +459,10 @@ ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* 
     set_weight_operand(h, d, W, L - 1);
     d.C = keep_logits ? h->Z : nullptr; d.ldc = h->ldz; d.alpha = 1.f; d.beta = 0.f;
     d.epi = EPI_LOGITS; d.bias = b[L - 1]; d.labels = labels;
+    if (tg.T) {         // the output deltas dE/dz go where the logits would, as a pair in 3xTF32 mode
+        d.epi = EPI_TANH_SSE; d.T = tg.T; d.ldt = tg.ldt;
+        d.C_lo = keep_logits ? h->Zlo : nullptr;
+    }
     d.stats = h->stats; d.stats_ld = h->stats_ld; d.zlabel = h->zlabel;
     d.splits = 1; d.k_per_split = d.K;
     const bool tc = use_tc(d, h->math);
@@ -460,13 +471,14 @@ ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* 
     if (tiles > h->stats_ld) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
     ulsnn_status_t st = timed_gemm(h, d, stream);
     if (st != ULSNN_OK) return st;
+    if (tg.T) return launch_rowsums(h->stats, h->stats_ld, tiles, n, h->loss_parts, accumulate, loss_out, stream);
     return launch_rowstats(h->stats, h->stats_ld, tiles, h->zlabel, n, h->lse, h->loss_parts, accumulate, loss_out, stream);
 }
 
 ulsnn_status_t check_call(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
-                          const int32_t* labels, int64_t n, double* loss_out) {
+                          const void* targets, int64_t n, double* loss_out) {
     if (!h || !W || !b || !loss_out || n < 0 || n > h->max_patterns) return ULSNN_ERR_INVALID_ARG;
-    if (n > 0 && (!X || !labels || ldx < h->sizes[0])) return ULSNN_ERR_INVALID_ARG;
+    if (n > 0 && (!X || !targets || ldx < h->sizes[0])) return ULSNN_ERR_INVALID_ARG;
     for (int l = 0; l < h->L; ++l) if (!W[l] || !b[l]) return ULSNN_ERR_INVALID_ARG;
     return ULSNN_OK;
 }
@@ -542,26 +554,28 @@ extern "C" ulsnn_status_t ulsnn_mlp_phase_times(ulsnn_mlp_t* h, int* n, float* m
     return ULSNN_OK;
 }
 
-extern "C" ulsnn_status_t ulsnn_mlp_forward_loss(ulsnn_mlp_t* h, const float* const* W, const float* const* b,
-                                                 const float* X, int64_t ldx, const int32_t* labels, int64_t n,
-                                                 double* loss_out, ulsnn_stream_t stream_) {
-    cudaStream_t stream = (cudaStream_t)stream_;
-    ulsnn_status_t st = check_call(h, W, b, X, ldx, labels, n, loss_out);
+namespace {
+
+ulsnn_status_t forward_call(ulsnn_mlp_t* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
+                            const Targets& tg, int64_t n, double* loss_out, cudaStream_t stream) {
+    ulsnn_status_t st = check_call(h, W, b, X, ldx, tg.T ? (const void*)tg.T : (const void*)tg.labels, n, loss_out);
     if (st != ULSNN_OK) return st;
+    if (tg.T && n > 0 && tg.ldt < h->sizes[h->L]) return ULSNN_ERR_INVALID_ARG;
     if ((st = check_arch()) != ULSNN_OK) return st;
     if (n == 0) return launch_zero_f64(loss_out, 1, stream);
-    return forward(h, W, b, X, ldx, labels, n, false, 0, loss_out, stream);
+    return forward(h, W, b, X, ldx, tg, n, false, 0, loss_out, stream);
 }
 
-extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const* W, const float* const* b,
-                                             const float* X, int64_t ldx, const int32_t* labels, int64_t n,
-                                             int accumulate, float* const* dW, float* const* db, double* loss_out,
-                                             ulsnn_stream_t stream_) {
-    cudaStream_t stream = (cudaStream_t)stream_;
-    ulsnn_status_t st = check_call(h, W, b, X, ldx, labels, n, loss_out);
+ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
+                             const Targets& tg, int64_t n, int accumulate, float* const* dW, float* const* db,
+                             double* loss_out, cudaStream_t stream) {
+    ulsnn_status_t st = check_call(h, W, b, X, ldx, tg.T ? (const void*)tg.T : (const void*)tg.labels, n, loss_out);
     if (st != ULSNN_OK) return st;
+    if (tg.T && n > 0 && tg.ldt < h->sizes[h->L]) return ULSNN_ERR_INVALID_ARG;
     if (!dW || !db) return ULSNN_ERR_INVALID_ARG;
     const int L = h->L;
+    const bool sse = tg.T != nullptr;
+    const int32_t* labels = tg.labels;
     for (int l = 0; l < L; ++l) if (!dW[l] || !db[l]) return ULSNN_ERR_INVALID_ARG;
     if ((st = check_arch()) != ULSNN_OK) return st;
     if (n == 0) {
@@ -572,16 +586,19 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
         }
         return launch_zero_f64(loss_out, 1, stream);
     }
-    if ((st = forward(h, W, b, X, ldx, labels, n, true, accumulate, loss_out, stream)) != ULSNN_OK) return st;
+    if ((st = forward(h, W, b, X, ldx, tg, n, true, accumulate, loss_out, stream)) != ULSNN_OK) return st;
 
     int64_t colsum_rows = 0;
     bool delta2_kept = false;       // the top delta product ran on the tensor-core engine and left delta_L in D2
     // Deltas of the hidden layers, top down: delta_l = (1 - H_l*H_l) * (delta_{l+1} W_{l+1})   (H_D of Section 4.2).
-    // delta_L is never stored: the kernels form softmax(z) - onehot from the logits as they load them.
+    // Softmax head: delta_L is not stored, the kernels form softmax(z) - onehot from the logits as they load them.
+    // Squared-error head: the output epilogue has written delta_L = dE/dz where the logits would be.
     for (int l = L - 1; l >= 1; --l) {
         GemmDesc d{};
         d.M = n; d.N = h->sizes[l]; d.K = h->sizes[l + 1];
-        if (l + 1 == L) {
+        if (l + 1 == L && sse) {
+            d.A = h->Z; d.A_lo = h->Zlo; d.a_sm = h->ldz;
+        } else if (l + 1 == L) {
             d.A = h->Z; d.a_sm = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 1;
             d.delta_out = h->D2; d.delta_out_lo = h->D2lo;      // kept for the weight-gradient product below
         }
@@ -593,7 +610,7 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
         d.epi = EPI_TANHP; d.Hm = h->H[l]; d.Hm_lo = h->Hlo[l]; d.ldh = h->ldh[l];
         d.colsum_part = (l == 1) ? h->colsum_parts : nullptr;
         d.splits = 1; d.k_per_split = d.K;
-        if (l + 1 == L) delta2_kept = use_tc(d, h->math) && tc_keeps_delta(d, h->math == ULSNN_MATH_3XTF32);
+        if (l + 1 == L && !sse) delta2_kept = use_tc(d, h->math) && tc_keeps_delta(d, h->math == ULSNN_MATH_3XTF32);
         if (l == 1) colsum_rows = ((n + 127) / 128) * (use_tc(d, h->math) ? tc_colsum_groups() : simt_colsum_groups());
         if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
     }
@@ -604,7 +621,8 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
     for (int w = L - 1; w >= 0; --w) {
         GemmDesc d{};
         d.M = h->sizes[w + 1]; d.N = h->sizes[w] + (w >= 1 ? 1 : 0); d.K = n;
-        if (w + 1 == L && delta2_kept) { d.A = h->D2; d.A_lo = h->D2lo; d.a_sk = h->ldz; }
+        if (w + 1 == L && sse) { d.A = h->Z; d.A_lo = h->Zlo; d.a_sk = h->ldz; }
+        else if (w + 1 == L && delta2_kept) { d.A = h->D2; d.A_lo = h->D2lo; d.a_sk = h->ldz; }
         else if (w + 1 == L) { d.A = h->Z; d.a_sk = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 0; }
         else            { d.A = h->D[w + 1]; d.a_sk = h->ldd[w + 1]; }
         d.a_sm = 1;
@@ -623,10 +641,44 @@ extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const*
     // bias gradient of the first layer: column sums of delta_1 (both engines use 128-row tiles)
     if (L >= 2) {
         st = launch_colsum_reduce(h->colsum_parts, colsum_rows, h->sizes[1], accumulate, db[0], stream);
+    } else if (sse) {
+        st = launch_matrix_colsum(h->Z, h->Zlo, h->ldz, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);
     } else {
         st = launch_delta_colsum(h->Z, h->ldz, h->lse, labels, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);
     }
     return st;
+}
+
+}  // namespace
+
+extern "C" ulsnn_status_t ulsnn_mlp_forward_loss(ulsnn_mlp_t* h, const float* const* W, const float* const* b,
+                                                 const float* X, int64_t ldx, const int32_t* labels, int64_t n,
+                                                 double* loss_out, ulsnn_stream_t stream) {
+    return forward_call(h, W, b, X, ldx, Targets{labels, nullptr, 0}, n, loss_out, (cudaStream_t)stream);
+}
+
+extern "C" ulsnn_status_t ulsnn_mlp_gradient(ulsnn_mlp_t* h, const float* const* W, const float* const* b,
+                                             const float* X, int64_t ldx, const int32_t* labels, int64_t n,
+                                             int accumulate, float* const* dW, float* const* db, double* loss_out,
+                                             ulsnn_stream_t stream) {
+    return gradient_call(h, W, b, X, ldx, Targets{labels, nullptr, 0}, n, accumulate, dW, db, loss_out, (cudaStream_t)stream);
+}
+
+extern "C" ulsnn_status_t ulsnn_mlp_forward_sse(ulsnn_mlp_t* h, const float* const* W, const float* const* b,
+                                                const float* X, int64_t ldx, const float* T, int64_t ldt, int64_t n,
+                                                double* loss_out, ulsnn_stream_t stream) {
+    if (n > 0 && !T) return ULSNN_ERR_INVALID_ARG;
+    static const float dummy = 0.f;
+    return forward_call(h, W, b, X, ldx, Targets{nullptr, T ? T : &dummy, ldt}, n, loss_out, (cudaStream_t)stream);
+}
+
+extern "C" ulsnn_status_t ulsnn_mlp_gradient_sse(ulsnn_mlp_t* h, const float* const* W, const float* const* b,
+                                                 const float* X, int64_t ldx, const float* T, int64_t ldt, int64_t n,
+                                                 int accumulate, float* const* dW, float* const* db, double* loss_out,
+                                                 ulsnn_stream_t stream) {
+    if (n > 0 && !T) return ULSNN_ERR_INVALID_ARG;
+    static const float dummy = 0.f;
+    return gradient_call(h, W, b, X, ldx, Targets{nullptr, T ? T : &dummy, ldt}, n, accumulate, dW, db, loss_out, (cudaStream_t)stream);
 }
 
 extern "C" ulsnn_status_t ulsnn_sgd_step(ulsnn_mlp_t* h, float* const* W, float* const* b,

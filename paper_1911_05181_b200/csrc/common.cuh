@@ -13,7 +13,9 @@ enum Epilogue : int {
     EPI_BIAS_TANH = 1,  // C = tanh(acc + bias[col]); optionally C[:, N] = 1         (Eq. 2 / H = tanh(X W^T))
     EPI_LOGITS    = 2,  // z = acc + bias[col]; per-(row, column-tile) softmax statistics, z at the label
     EPI_TANHP     = 3,  // C = (1 - h*h) * acc, h = Hm[row][col]; per-row-tile column sums (H_D of Section 4.2)
-    EPI_PARTIAL   = 4   // split-K slice: raw accumulator into partials[slice]
+    EPI_PARTIAL   = 4,  // split-K slice: raw accumulator into partials[slice]
+    EPI_TANH_SSE  = 5   // the paper's output layer (Eqs. 1, 3): y = tanh(acc + bias); per-(row, column-tile) sums of
+                        // (y - t)^2; C = 2 (y - t)(1 - y^2) = dE/dz (optionally as a (hi, lo) pair)
 };
 
 // One product D = op(A) op(B) plus its fused epilogue; both engines (FFMA and tcgen05) take this.
@@ -26,7 +28,7 @@ struct GemmDesc {
     // then needs no operand pass for it in 3xTF32 mode; the FFMA engine adds the two.
     const float* A_lo; const float* B_lo;
     float* C; int64_t ldc;
-    float* C_lo;              // BIAS_TANH: not null -> C gets tf32_rn(h) and C_lo the rounded remainder (same ldc)
+    float* C_lo;              // BIAS_TANH, TANH_SSE: not null -> C gets tf32_rn(v) and C_lo the rounded remainder (same ldc)
     float alpha, beta;
     int epi;
     // epilogue operands
@@ -36,7 +38,8 @@ struct GemmDesc {
     const float* Hm_lo;       // TANHP: not null -> h = Hm + Hm_lo
     float* colsum_part;       // TANHP: [row_tiles * groups][N] partial column sums (may be null)
     const int32_t* labels;    // LOGITS and the A transform: label of each pattern
-    float2* stats; int64_t stats_ld;     // LOGITS: stats[row*stats_ld + col_tile] = (max, sum exp(z - max))
+    const float* T; int64_t ldt;         // TANH_SSE: targets [M x N], rows ldt apart
+    float2* stats; int64_t stats_ld;     // LOGITS: stats[row*stats_ld + col_tile] = (max, sum exp(z - max)); TANH_SSE: (0, sum (y-t)^2)
     float* zlabel;            // LOGITS: z[row][label[row]]
     // A transform: the stored operand holds logits z; the product uses softmax(z) - onehot(label)
     int a_transform;
@@ -89,6 +92,12 @@ ulsnn_status_t launch_rowstats(const float2* stats, int64_t stats_ld, int tiles,
                                float* lse, double* block_partials, int accumulate, double* loss_out,
                                cudaStream_t stream);
 int rowstats_blocks(int64_t n);
+// loss = sum_p sum_t stats[p*stats_ld + t].y in a fixed order, in double (the squared-error head)
+ulsnn_status_t launch_rowsums(const float2* stats, int64_t stats_ld, int tiles, int64_t n, double* block_partials,
+                              int accumulate, double* loss_out, cudaStream_t stream);
+// out[j] = sum_p (A[p*lda + j] + A_lo[p*lda + j])  (A_lo may be null), rows added in a fixed order
+ulsnn_status_t launch_matrix_colsum(const float* A, const float* A_lo, int64_t lda, int64_t n, int64_t cols, float* parts,
+                                    int accumulate, float* out, cudaStream_t stream);
 // db[j] = sum_p softmax(z_p)_j - [label_p == j]   (only for networks without a hidden layer)
 ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* lse, const int32_t* labels,
                                    int64_t n, int64_t n_classes, float* parts, int accumulate, float* out,

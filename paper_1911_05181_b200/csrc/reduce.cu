@@ -79,6 +79,22 @@ __global__ void rowstats_kernel(const float2* __restrict__ stats, int64_t stats_
     if (threadIdx.x == 0) block_partials[blockIdx.x] = red[0];
 }
 
+// squared-error head: one thread per pattern adds its per-tile sums in tile order, then a fixed tree over the block
+__global__ void rowsums_kernel(const float2* __restrict__ stats, int64_t stats_ld, int tiles, int64_t n,
+                               double* __restrict__ block_partials) {
+    __shared__ double red[RS_THREADS];
+    const int64_t p = (int64_t)blockIdx.x * RS_THREADS + threadIdx.x;
+    double term = 0.0;
+    if (p < n) for (int t = 0; t < tiles; ++t) term += (double)stats[p * stats_ld + t].y;
+    red[threadIdx.x] = term;
+    __syncthreads();
+    for (int o = RS_THREADS / 2; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) block_partials[blockIdx.x] = red[0];
+}
+
 __global__ void loss_final_kernel(const double* __restrict__ block_partials, int nblocks, int accumulate,
                                   double* __restrict__ loss_out) {
     // a single thread: a few hundred additions in index order
@@ -88,6 +104,16 @@ __global__ void loss_final_kernel(const double* __restrict__ block_partials, int
 }
 
 constexpr int DC_ROWS = 1024;   // patterns per partial row of the delta column sum
+
+__global__ void matrix_colsum_kernel(const float* __restrict__ A, const float* __restrict__ A_lo, int64_t lda, int64_t n,
+                                     int64_t cols, float* __restrict__ parts) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= cols) return;
+    const int64_t p0 = (int64_t)blockIdx.y * DC_ROWS, p1 = min(n, p0 + DC_ROWS);
+    float s = 0.f;
+    for (int64_t p = p0; p < p1; ++p) s += A[p * lda + j] + (A_lo ? A_lo[p * lda + j] : 0.f);
+    parts[(int64_t)blockIdx.y * cols + j] = s;
+}
 
 __global__ void delta_colsum_kernel(const float* __restrict__ Z, int64_t ldz, const float* __restrict__ lse,
                                     const int32_t* __restrict__ labels, int64_t n, int64_t n_classes,
@@ -197,6 +223,32 @@ ulsnn_status_t launch_rowstats(const float2* stats, int64_t stats_ld, int tiles,
     loss_final_kernel<<<1, 1, 0, stream>>>(block_partials, nb, accumulate, loss_out);
     ulsnn::count_launch(2);
     return cuda_ok(cudaGetLastError());
+}
+
+ulsnn_status_t launch_rowsums(const float2* stats, int64_t stats_ld, int tiles, int64_t n, double* block_partials,
+                              int accumulate, double* loss_out, cudaStream_t stream) {
+    const int nb = rowstats_blocks(n);
+    if (nb > 0) {
+        rowsums_kernel<<<nb, RS_THREADS, 0, stream>>>(stats, stats_ld, tiles, n, block_partials);
+        ulsnn::count_launch(2);
+        if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
+    }
+    loss_final_kernel<<<1, 1, 0, stream>>>(block_partials, nb, accumulate, loss_out);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+ulsnn_status_t launch_matrix_colsum(const float* A, const float* A_lo, int64_t lda, int64_t n, int64_t cols, float* parts,
+                                    int accumulate, float* out, cudaStream_t stream) {
+    const int tiles = (int)((n + DC_ROWS - 1) / DC_ROWS);
+    if (tiles > 65535) return ULSNN_ERR_TOO_LARGE;
+    if (tiles > 0) {
+        dim3 grid((unsigned)((cols + 127) / 128), (unsigned)tiles);
+        matrix_colsum_kernel<<<grid, 128, 0, stream>>>(A, A_lo, lda, n, cols, parts);
+        ulsnn::count_launch(2);
+        if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
+    }
+    return launch_colsum_reduce(parts, tiles, cols, accumulate, out, stream);
 }
 
 int delta_colsum_tiles(int64_t n) { return (int)((n + DC_ROWS - 1) / DC_ROWS); }

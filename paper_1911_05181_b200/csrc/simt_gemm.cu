@@ -184,6 +184,36 @@ __global__ void __launch_bounds__(NT) simt_gemm_kernel(const GemmDesc d) {
                 }
             }
         }
+    } else if (EPI == EPI_TANH_SSE) {
+        // Threads tx = 0..15 of one ty share a row and sit in one half-warp (as in the logits epilogue).
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int64_t r = row_of(i);
+            const bool rv = r < d.M;
+            float s = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int64_t c = col_of(j);
+                if (rv && c < d.N) {
+                    const float y = tanhf(acc[i][j] + __ldg(d.bias + c));
+                    const float e = y - __ldg(d.T + r * d.ldt + c);
+                    s += e * e;
+                    if (d.C) {
+                        const float g = 2.f * e * (1.f - y * y);
+                        if (d.C_lo) {
+                            const float hi = __uint_as_float((__float_as_uint(g) + 0x1000u) & 0xFFFFE000u);
+                            d.C[r * d.ldc + c] = hi;
+                            d.C_lo[r * d.ldc + c] = __uint_as_float((__float_as_uint(g - hi) + 0x1000u) & 0xFFFFE000u);
+                        } else {
+                            d.C[r * d.ldc + c] = g;
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int o = 8; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (rv && tx == 0) d.stats[r * d.stats_ld + blockIdx.y] = make_float2(0.f, s);
+        }
     } else if (EPI == EPI_TANHP) {
         float cs[8];
 #pragma unroll
@@ -247,6 +277,7 @@ ulsnn_status_t simt_gemm_launch(const GemmDesc& d, cudaStream_t stream) {
         case EPI_LOGITS:    return tr ? ULSNN_ERR_INVALID_ARG : launch<EPI_LOGITS, false>(d, stream);
         case EPI_TANHP:     return tr ? launch<EPI_TANHP, true>(d, stream) : launch<EPI_TANHP, false>(d, stream);
         case EPI_PARTIAL:   return tr ? launch<EPI_PARTIAL, true>(d, stream) : launch<EPI_PARTIAL, false>(d, stream);
+        case EPI_TANH_SSE:  return tr ? ULSNN_ERR_INVALID_ARG : launch<EPI_TANH_SSE, false>(d, stream);
     }
     return ULSNN_ERR_INVALID_ARG;
 }

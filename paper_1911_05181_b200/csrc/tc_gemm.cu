@@ -611,7 +611,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint8_t* stg = epi_scratch + ew * (2 * EPI_STAGE_BYTES);     // two 32x32 store-staging blocks of this warp
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
         const bool c_vec = ((((uintptr_t)d.C) & 15) == 0) && ((d.ldc & 3) == 0);
-        const bool bias_vec = (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) && ((((uintptr_t)d.bias) & 15) == 0);
+        const bool bias_vec = (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS || EPI == EPI_TANH_SSE) && ((((uintptr_t)d.bias) & 15) == 0);
+        const bool t_vec = (EPI == EPI_TANH_SSE) && ((((uintptr_t)d.T) & 15) == 0) && ((d.ldt & 3) == 0);
         const bool h_vec = (EPI == EPI_TANHP) && ((((uintptr_t)d.Hm) & 15) == 0) && ((((uintptr_t)d.Hm_lo) & 15) == 0) && ((d.ldh & 3) == 0);
         uint32_t tile_i = 0, stg_i = 0;
         uint32_t reads[2] = {0, 0};             // how often each TMEM region has been waited for
@@ -685,7 +686,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = d.alpha * v[j];
                     }
-                } else if (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) {
+                } else if (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS || EPI == EPI_TANH_SSE) {
                     if (bias_vec && full) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
@@ -699,6 +700,35 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (EPI == EPI_BIAS_TANH) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = tanhf(v[j]);
+                    } else if (EPI == EPI_TANH_SSE) {
+                        // Eqs. 1 and 3: y = tanh(z), E += (y - t)^2, stored value dE/dz = 2 (y - t)(1 - y^2)
+                        float t[32];
+                        if (rv) {
+                            const float* tp = d.T + r * d.ldt + c0;
+                            if (t_vec && full) {
+#pragma unroll
+                                for (int j = 0; j < 32; j += 4) {
+                                    const float4 q4 = __ldg(reinterpret_cast<const float4*>(tp + j));
+                                    t[j] = q4.x; t[j + 1] = q4.y; t[j + 2] = q4.z; t[j + 3] = q4.w;
+                                }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) t[j] = (j < nvalid) ? __ldg(tp + j) : 0.f;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) t[j] = 0.f;
+                        }
+                        float s = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float y = tanhf(v[j]);
+                            const float e = (j < nvalid) ? y - t[j] : 0.f;
+                            s += e * e;
+                            v[j] = 2.f * e * (1.f - y * y);
+                        }
+                        run_s += s;
+                        do_store = d.C != nullptr;
                     } else {
                         float cm = -INFINITY;
 #pragma unroll
@@ -781,7 +811,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (do_store) {
                     if (EPI == EPI_PARTIAL) {
                         store_block(v, &map_c, d.partials + (int64_t)sp * d.M * d.ldp, d.ldp);
-                    } else if (EPI == EPI_BIAS_TANH && p.c_pair) {
+                    } else if ((EPI == EPI_BIAS_TANH || EPI == EPI_TANH_SSE) && p.c_pair) {
                         float lo[32];
 #pragma unroll
                         for (int j = 0; j < 32; ++j) { const float h = to_tf32(v[j]); lo[j] = to_tf32(v[j] - h); v[j] = h; }
@@ -805,6 +835,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             __syncwarp();
             if (lane == 0) { if (CG == 2 && rank == 1) signal_rank0(smem_u32(&ctrl->free_sink[acc][ew]), smem_u32(&ctrl->reg_free[acc])); else mbar_arrive(smem_u32(&ctrl->reg_free[acc])); }
 
+            if (EPI == EPI_TANH_SSE && rv) d.stats[r * d.stats_ld + nt] = make_float2(0.f, run_s);
             if (EPI == EPI_LOGITS && rv) {
                 d.stats[r * d.stats_ld + nt] = make_float2(run_m, run_s);
                 if (have_zl) d.zlabel[r] = zl;
@@ -1128,7 +1159,7 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     if (!map_of_a(&m.a, d.A) || !map_of_b(&m.b, d.B)) return ULSNN_ERR_CUDA;
     if (p.a_pre && !map_of_a(&m.a_lo, d.A_lo)) return ULSNN_ERR_CUDA;
     if (p.b_pre && !map_of_b(&m.b_lo, d.B_lo)) return ULSNN_ERR_CUDA;
-    p.c_pair = (d.epi == EPI_BIAS_TANH && d.C_lo) ? 1 : 0;
+    p.c_pair = ((d.epi == EPI_BIAS_TANH || d.epi == EPI_TANH_SSE) && d.C_lo) ? 1 : 0;
     // deltas kept for a later product: the transformed K-major A tile in shared memory is exactly one TMA box
     if (tc_keeps_delta(d, three_x)) {
         p.d_out = make_map(&m.d, d.delta_out, d.K, d.M, d.a_sm, BK, BM, false) &&
@@ -1142,7 +1173,7 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
         // A TMA store clips a row at the next 16-byte boundary past the matrix edge, so a width that is not a multiple
         // of four spills up to three floats into the row's padding.  That padding is scratch in the library's own
         // logit and delta buffers; it belongs to the caller in C, and it is the ones column in an activation buffer.
-        const bool pad_is_scratch = d.epi == EPI_LOGITS || d.epi == EPI_TANHP;
+        const bool pad_is_scratch = d.epi == EPI_LOGITS || d.epi == EPI_TANHP || d.epi == EPI_TANH_SSE;
         if ((d.N & 3) == 0 || pad_is_scratch) p.c_tma = make_store_map(&m.c, d.C, d.N, d.M, d.ldc, 1) ? 1 : 0;
         if (p.c_tma && p.c_pair)
             p.c_tma = ((((uintptr_t)d.C_lo) & 15) == 0 && make_store_map(&m.c_lo, d.C_lo, d.N, d.M, d.ldc, 1)) ? 1 : 0;
@@ -1157,6 +1188,7 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
         case EPI_LOGITS:    return launch_cg<EPI_LOGITS>(cg, m, p, smem_bytes, grid, stream);
         case EPI_TANHP:     return launch_cg<EPI_TANHP>(cg, m, p, smem_bytes, grid, stream);
         case EPI_PARTIAL:   return launch_cg<EPI_PARTIAL>(cg, m, p, smem_bytes, grid, stream);
+        case EPI_TANH_SSE:  return launch_cg<EPI_TANH_SSE>(cg, m, p, smem_bytes, grid, stream);
     }
     return ULSNN_ERR_INVALID_ARG;
 }

@@ -29,6 +29,7 @@ _MIX2 = np.uint64(0x94D049BB133111EB)
 # Tensor ids used by every config (kept here so host and device agree).
 TID_X = 1
 TID_LABELS = 2
+TID_TARGETS = 3
 TID_W0 = 16        # W_l uses TID_W0 + 2*l, b_l uses TID_W0 + 2*l + 1
 TID_GEMM_A = 100
 TID_GEMM_B = 101
@@ -103,6 +104,18 @@ def mlp_batch(seed: int, sizes, n_patterns: int, offset: int = 0):
     X = uniform01(seed, TID_X, n_patterns * n0, offset * n0).reshape(n_patterns, n0)
     y = labels(seed, TID_LABELS, n_patterns, nL, offset)
     return X, y
+
+
+def mlp_targets(seed: int, sizes, n_patterns: int, offset: int = 0, coded: bool = False):
+    """Dense target matrix T [n_patterns, n_L] for the squared-error head: uniform[-1,1), or, with coded=True,
+    the +1 / -1 code of the pattern's label (one output unit per class)."""
+    nL = int(sizes[-1])
+    if coded:
+        y = labels(seed, TID_LABELS, n_patterns, nL, offset)
+        T = np.full((n_patterns, nL), -1.0, dtype=np.float32)
+        T[np.arange(n_patterns), y] = 1.0
+        return T
+    return uniform_pm1(seed, TID_TARGETS, n_patterns * nL, offset * nL).reshape(n_patterns, nL)
 
 
 def gemm_operands(seed: int, rows_a: int, cols_a: int, rows_b: int, cols_b: int,
