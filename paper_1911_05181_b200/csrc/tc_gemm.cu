@@ -1,29 +1,34 @@
 // tcgen05 engine: TF32 tensor-core GEMM for sm_100a with TMEM accumulators, TMA-fed shared-memory ring,
-// an on-chip hi/lo operand split for the error-compensated 3xTF32 mode, and the fused epilogues.
+// the error-compensated 3xTF32 mode (operands as TF32 hi/lo pairs, split on chip or loaded as stored pairs),
+// and the fused epilogues.
 //
 // One persistent CTA per SM, 14 warps with fixed roles:
-//   warp 0      TMA producer      global -> 128B-swizzled shared-memory stages (cp.async.bulk.tensor, no multicast)
-//   warp 1      MMA issuer        one thread issues tcgen05.mma.kind::tf32 (128 x BN x 8 per instruction)
+//   warp 0      TMA producer      global -> swizzled shared-memory stages (cp.async.bulk.tensor, no multicast);
+//                                 also stores transformed A stages back to global memory when deltas are kept
+//   warp 1      product issuer    all lanes run the loop, an elected lane issues tcgen05.mma.kind::tf32 and the
+//                                 commits (in the second CTA of a pair: relays "stage ready" to the first)
 //   warps 2-5   epilogue          tcgen05.ld of the 128 x BN fp32 accumulator (one row per thread), fused math, then
 //                                 32x32 blocks staged in swizzled shared memory and written with TMA stores
 //                                 (whole 128-byte lines, edges clipped by the tensor map)
-//   warps 6-13  operand pass      only in 3xTF32 mode or when A is formed from logits: reads a landed stage,
-//                                 rewrites it as hi = tf32_rn(x) and writes lo = tf32(x - hi) beside it.  (The
-//                                 tensor core ignores the low 13 mantissa bits of an fp32 word, so the landed tile
-//                                 could serve as hi = trunc(x) unchanged; the lo parts then all have the sign of x
-//                                 and the accumulator's truncation no longer averages out: measured 2.4x the error.)
+//   warps 6-13  operand pass      for operands that do not arrive as stored pairs (3xTF32), or when A is formed
+//                                 from logits: reads a landed stage, rewrites it as hi = tf32_rn(x) and writes
+//                                 lo = tf32_rn(x - hi) beside it
+// Tiles: 128 x BN (BN <= 256) by one CTA, or 256 x BN by the two CTAs of a cluster (tcgen05 cta_group::2): each
+// CTA holds its 128 rows of A, half of the B tile and its 128 rows of the accumulator; CTA 0 issues the products.
+// CTA 1 signals CTA 0 with asynchronous stores that complete transaction bytes on CTA 0's barriers; CTA 0 answers
+// through multicast tcgen05.commit.
 // TMEM holds two 256-column accumulator regions.  A tile's total lives in one of them, so its epilogue overlaps
 // the products of the next tile, which uses the other.  The tensor core adds into an fp32 accumulator with
-// truncation, a bias that grows with the number of instructions chained on one accumulator; in 3xTF32 mode the
+// truncation, an error that grows with the number of instructions chained on one accumulator; in 3xTF32 mode the
 // K loop is therefore cut into chunks of 256: each chunk starts a fresh accumulator in the second region and
 // the epilogue warps add it (round-to-nearest) into the tile's total, kept in TMEM.
 // 3xTF32: D += lo_a*hi_b; D += hi_a*lo_b; D += hi_a*hi_b (small terms first).
 // MN-major fp32 operands use the 128B swizzle with 32-byte atoms (the only one the tensor core transposes
-// for 32-bit types); K-major operands the plain 128B swizzle.
+// for 32-bit types); K-major operands the plain 128B swizzle (64B when BK = 16).
 // Both operands may be K-major or MN-major in memory (transpose bits of the instruction descriptor), so the
 // four forms of Section 3.1 and the three product shapes of Section 4.2 are one kernel.
-// Every wait is bounded: on expiry the CTA raises an abort flag, records DEV_TIMEOUT in the device status
-// word, drains and frees its TMEM.
+// Every wait on an mbarrier is bounded: on expiry the CTA raises an abort flag, records DEV_TIMEOUT in the
+// device status word, drains and frees its TMEM.
 #include "common.cuh"
 #include <cuda.h>
 #include <math.h>
