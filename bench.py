@@ -290,10 +290,53 @@ def main():
         step(X, y, host=(Xh, yh))
         loss_h.copy_(loss, non_blocking=True)
 
-    for _ in range(2):
-        e2e_step()
-    reset_params()
-    ms_e2e = timed(e2e_step, args.steps)
+    if len(starts) == 1:
+        # Double-buffered: while step i computes on one device buffer, a copy stream brings step i+1's batch from
+        # pinned host memory into the other.  Every step still pays for its own host-to-device copy and reads its
+        # loss back; the timed region starts before the first copy and ends after the last read-back.
+        copy_stream = torch.cuda.Stream()
+        bufs = [(X, y), (torch.empty_like(X), torch.empty_like(y))]
+        copied = [torch.cuda.Event() for _ in range(2)]
+        freed = [torch.cuda.Event() for _ in range(2)]
+
+        def prefetch(i):
+            with torch.cuda.stream(copy_stream):
+                copy_stream.wait_event(freed[i % 2])
+                bufs[i % 2][0].copy_(Xh, non_blocking=True); bufs[i % 2][1].copy_(yh, non_blocking=True)
+                copied[i % 2].record(copy_stream)
+
+        def run_e2e(steps):
+            for ev in freed:
+                ev.record(stream)
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            barrier()
+            e0.record(stream)
+            copy_stream.wait_event(e0)
+            prefetch(0)
+            for i in range(steps):
+                stream.wait_event(copied[i % 2])
+                if i + 1 < steps:
+                    prefetch(i + 1)
+                step(*bufs[i % 2])
+                freed[i % 2].record(stream)
+                loss_h.copy_(loss, non_blocking=True)
+            e1.record(stream)
+            barrier()
+            ms = e0.elapsed_time(e1)
+            if world > 1:
+                t = torch.tensor([ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = float(t.item())
+            return ms / steps
+
+        run_e2e(2)
+        reset_params()
+        ms_e2e = run_e2e(args.steps)
+        e2e_mode = "double-buffered host-to-device copies on a second stream"
+    else:
+        for _ in range(2):
+            e2e_step()
+        reset_params()
+        ms_e2e = timed(e2e_step, args.steps)
+        e2e_mode = "each chunk copied from pinned host memory right before it is evaluated"
 
     gflop_step = flops.gradient_flops(sizes, batch) * world / 1e9
     value = gflop_step / (ms_step * 1e-3)
@@ -349,7 +392,7 @@ def main():
                    "step": "gradient evaluation + W -= lr*grad, lr = 1e-3 / global_batch"},
         "patterns_per_s": batch * world / (ms_step * 1e-3),
         "pct_of_tf32_peak": None,
-        "e2e": {"value": e2e_value, "unit": "GFLOP/s", "ms_per_step": ms_e2e,
+        "e2e": {"value": e2e_value, "unit": "GFLOP/s", "ms_per_step": ms_e2e, "how": e2e_mode,
                 "h2d_bytes_per_step": Xh.numel() * 4 + yh.numel() * 4, "d2h_bytes_per_step": 8},
         "gpu_launches": int(launches),
         "launch_kinds": {k: int(c1[k] - c0[k]) for k in c1},
