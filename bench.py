@@ -140,7 +140,7 @@ def run_reference(args):
     sizes, batch, seed = WORKLOADS[args.workload]
     if args.patterns > 0:
         batch = args.patterns
-    n_sample = min(batch, 2048 if args.workload != "config5" else 128)
+    n_sample = min(batch, 1024 if args.workload != "config5" else 128)
     Ws, bs = si.mlp_params(seed, sizes)
     X, y = si.mlp_batch(seed, sizes, n_sample)
     for _ in range(args.warmup):
@@ -168,6 +168,67 @@ def run_reference(args):
     return 0
 
 
+SGEMM_SWEEP = [  # (transA, transB, M, N, K): the standalone-SGEMM configuration (Section 3.4's experiment, restaged)
+    ("N", "N", 256, 256, 256), ("N", "N", 1024, 1024, 1024), ("N", "N", 4096, 4096, 4096), ("N", "N", 8192, 8192, 8192),
+    ("N", "T", 4096, 4096, 4096), ("T", "N", 4096, 4096, 4096), ("T", "T", 4096, 4096, 4096),
+    ("N", "T", 65536, 480, 400), ("N", "T", 65536, 3204, 480), ("T", "N", 480, 3204, 65536),
+]
+
+
+def run_sgemm_sweep(args):
+    """--workload sgemm: C = A*B (alpha 1, beta 0) over the sweep, device-resident operands uniform [-1,1), seed 1.
+    N = 3204 stands in for 3203 (a packed leading dimension of 3203 floats cannot be addressed by TMA and goes to
+    the FFMA engine).  Prints one JSON line; `value` is the 8192^3 rate."""
+    import torch
+    import synth_inputs as si
+    from paper_1911_05181_b200 import binding as ul
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return 0
+    math_mode = MATH[args.math]
+    peaks = load_peaks()
+    tf32_peak = peaks["bf16_tflops_sustained"] * NOMINAL_TF32_OVER_BF16
+    mult = 3.0 if args.math == "3xtf32" else 1.0
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")          # > L2: written between timed calls
+    rows = []
+    for ta, tb, M, N, K in SGEMM_SWEEP:
+        ra, ca = (K, M) if ta == "T" else (M, K)
+        rb, cb = (N, K) if tb == "T" else (K, N)
+        A = torch.empty(ra, ca, device="cuda"); B = torch.empty(rb, cb, device="cuda"); C = torch.empty(M, N, device="cuda")
+        ul.fill_uniform(A, A.numel(), 1, si.TID_GEMM_A, 0, 1); ul.fill_uniform(B, B.numel(), 1, si.TID_GEMM_B, 0, 1)
+        nbytes = ul.sgemm_workspace_bytes(ta, tb, M, N, K, math_mode)
+        ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+        wp = (ws.data_ptr() + 255) // 256 * 256
+
+        def call():
+            ul.sgemm_ex(ta, tb, M, N, K, 1.0, A, ca, B, cb, 0.0, C, N, math_mode, wp if nbytes else None, nbytes)
+
+        for _ in range(3):
+            call()
+        reps = 20 if M * N * K < (1 << 34) else 8
+        times = []
+        for _ in range(reps):
+            flush.fill_(1)                                                     # cold L2, as the paper flushed its caches
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream); call(); e1.record(stream)
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms = statistics.median(times)
+        tf = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+        rows.append({"form": ta + tb, "M": M, "N": N, "K": K, "ms": round(ms, 4), "logical_tflops": round(tf, 2),
+                     "tensor_pipe_frac_of_measured": round(mult * tf / tf32_peak, 3) if args.math != "simt" else None})
+    big = [r for r in rows if r["M"] == 8192][0]
+    line = {"metric": "sgemm_gflops", "value": big["logical_tflops"] * 1e3, "unit": "GFLOP/s", "n_gpus": 1, "steps": 8,
+            "warmup": 3, "ms_per_step": big["ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "sgemm sweep (alpha 1, beta 0, uniform [-1,1), seed 1); value = NN 8192^3", "math": args.math,
+                       "l2": "a 256 MB buffer is overwritten between timed calls"},
+            "sweep": rows, "peak_tflops": tf32_peak, "gpu_launches": int(sum(ul.launch_counts().values()))}
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -175,7 +236,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--math", default="3xtf32", choices=sorted(MATH))
-    ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS) + ["sgemm"])
     ap.add_argument("--head", default="softmax", choices=["softmax", "sse"],
                     help="softmax + cross-entropy on labels (the benchmark's workload) or the paper's tanh outputs with "
                          "summed squared error on a dense target matrix")
@@ -183,6 +244,8 @@ def main():
     ap.add_argument("--patterns", type=int, default=0,
                     help="patterns per GPU instead of the workload's own count (for profiler captures of a smaller case)")
     args = ap.parse_args()
+    if args.workload == "sgemm":
+        return run_sgemm_sweep(args) if args.impl == "ours" else 0
     if args.impl == "reference":
         return run_reference(args)
 
