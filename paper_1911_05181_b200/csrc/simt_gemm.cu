@@ -36,7 +36,7 @@ __device__ __forceinline__ float load_b(const GemmDesc& d, int64_t k, int64_t j,
 }
 
 template <int EPI, bool TRANSFORM>
-__global__ void __launch_bounds__(NT) simt_gemm_kernel(const GemmDesc d) {
+__global__ void __launch_bounds__(NT, 2) simt_gemm_kernel(const GemmDesc d) {
     __shared__ Tile sm;
     const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
     const int64_t m0 = (int64_t)blockIdx.x * BM, n0 = (int64_t)blockIdx.y * BN;
@@ -50,25 +50,92 @@ __global__ void __launch_bounds__(NT) simt_gemm_kernel(const GemmDesc d) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
 
+    // Staging of the next k tile in registers.  When an operand tile lies inside the matrix and its rows are 16-byte
+    // aligned, each thread fetches two float4 along the contiguous direction; otherwise eight guarded scalars.
+    const bool a_vec = !TRANSFORM && !d.A_lo && ((((uintptr_t)d.A) & 15) == 0) &&
+                       (a_kc ? ((d.a_sm & 3) == 0) : ((d.a_sk & 3) == 0)) && (m0 + BM <= d.M);
+    const bool b_vec = !d.B_lo && ((((uintptr_t)d.B) & 15) == 0) &&
+                       (b_nc ? ((d.b_sk & 3) == 0) : ((d.b_sn & 3) == 0)) && (n0 + BN <= d.N);
     float ra[8], rb[8];
+    bool va = false, vb = false;        // how the staged registers were fetched
     auto fetch = [&](int64_t k0) {
+        const bool kfull = k0 + BK <= kend;
+        va = a_vec && kfull; vb = b_vec && kfull;
+        if (va) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int e = t + NT * i;
-            const int am = a_kc ? (e >> 4) : (e & 127), ak = a_kc ? (e & 15) : (e >> 7);
-            ra[i] = load_a<TRANSFORM>(d, m0 + am, k0 + ak, kend);
-            const int bn = b_nc ? (e & 127) : (e >> 4), bk = b_nc ? (e >> 7) : (e & 15);
-            rb[i] = load_b(d, k0 + bk, n0 + bn, kend);
+            for (int i = 0; i < 2; ++i) {
+                const int e = t + NT * i;                                   // float4 index in the 128 x 16 tile
+                const int am = a_kc ? (e >> 2) : ((e & 31) << 2), ak = a_kc ? ((e & 3) << 2) : (e >> 5);
+                const float4 v = __ldg(reinterpret_cast<const float4*>(d.A + (m0 + am) * d.a_sm + (k0 + ak) * d.a_sk));
+                ra[4 * i] = v.x; ra[4 * i + 1] = v.y; ra[4 * i + 2] = v.z; ra[4 * i + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int e = t + NT * i;
+                const int am = a_kc ? (e >> 4) : (e & 127), ak = a_kc ? (e & 15) : (e >> 7);
+                ra[i] = load_a<TRANSFORM>(d, m0 + am, k0 + ak, kend);
+            }
+        }
+        if (vb) {
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int e = t + NT * i;
+                const int bn = b_nc ? ((e & 31) << 2) : (e >> 2), bk = b_nc ? (e >> 5) : ((e & 3) << 2);
+                const float4 v = __ldg(reinterpret_cast<const float4*>(d.B + (k0 + bk) * d.b_sk + (n0 + bn) * d.b_sn));
+                rb[4 * i] = v.x; rb[4 * i + 1] = v.y; rb[4 * i + 2] = v.z; rb[4 * i + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int e = t + NT * i;
+                const int bn = b_nc ? (e & 127) : (e >> 4), bk = b_nc ? (e >> 7) : (e & 15);
+                rb[i] = load_b(d, k0 + bk, n0 + bn, kend);
+            }
         }
     };
     auto stash = [&](int buf) {
+        if (va) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int e = t + NT * i;
-            const int am = a_kc ? (e >> 4) : (e & 127), ak = a_kc ? (e & 15) : (e >> 7);
-            sm.a[buf][ak][am] = ra[i];
-            const int bn = b_nc ? (e & 127) : (e >> 4), bk = b_nc ? (e >> 7) : (e & 15);
-            sm.b[buf][bk][bn] = rb[i];
+            for (int i = 0; i < 2; ++i) {
+                const int e = t + NT * i;
+                if (a_kc) {         // four consecutive k of one row: a transposing store
+                    const int am = e >> 2, ak = (e & 3) << 2;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) sm.a[buf][ak + j][am] = ra[4 * i + j];
+                } else {            // four consecutive rows of one k
+                    const int am = (e & 31) << 2, ak = e >> 5;
+                    *reinterpret_cast<float4*>(&sm.a[buf][ak][am]) = make_float4(ra[4 * i], ra[4 * i + 1], ra[4 * i + 2], ra[4 * i + 3]);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int e = t + NT * i;
+                const int am = a_kc ? (e >> 4) : (e & 127), ak = a_kc ? (e & 15) : (e >> 7);
+                sm.a[buf][ak][am] = ra[i];
+            }
+        }
+        if (vb) {
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int e = t + NT * i;
+                if (b_nc) {
+                    const int bn = (e & 31) << 2, bk = e >> 5;
+                    *reinterpret_cast<float4*>(&sm.b[buf][bk][bn]) = make_float4(rb[4 * i], rb[4 * i + 1], rb[4 * i + 2], rb[4 * i + 3]);
+                } else {
+                    const int bn = e >> 2, bk = (e & 3) << 2;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) sm.b[buf][bk + j][bn] = rb[4 * i + j];
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int e = t + NT * i;
+                const int bn = b_nc ? (e & 127) : (e >> 4), bk = b_nc ? (e >> 7) : (e & 15);
+                sm.b[buf][bk][bn] = rb[i];
+            }
         }
     };
 
