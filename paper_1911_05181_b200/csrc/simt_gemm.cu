@@ -52,8 +52,9 @@ __global__ void __launch_bounds__(NT, 2) simt_gemm_kernel(const GemmDesc d) {
 
     // Staging of the next k tile in registers.  When an operand tile lies inside the matrix and its rows are 16-byte
     // aligned, each thread fetches two float4 along the contiguous direction; otherwise eight guarded scalars.
-    const bool a_vec = !TRANSFORM && !d.A_lo && ((((uintptr_t)d.A) & 15) == 0) &&
-                       (a_kc ? ((d.a_sm & 3) == 0) : ((d.a_sk & 3) == 0)) && (m0 + BM <= d.M);
+    const bool a_vec = !d.A_lo && ((((uintptr_t)d.A) & 15) == 0) &&
+                       (a_kc ? ((d.a_sm & 3) == 0) : ((d.a_sk & 3) == 0)) && (m0 + BM <= d.M) &&
+                       (!TRANSFORM || a_kc == (d.a_pattern_is_m != 0));      // logits: the class is the contiguous index
     const bool b_vec = !d.B_lo && ((((uintptr_t)d.B) & 15) == 0) &&
                        (b_nc ? ((d.b_sk & 3) == 0) : ((d.b_sn & 3) == 0)) && (n0 + BN <= d.N);
     float ra[8], rb[8];
@@ -68,6 +69,15 @@ __global__ void __launch_bounds__(NT, 2) simt_gemm_kernel(const GemmDesc d) {
                 const int am = a_kc ? (e >> 2) : ((e & 31) << 2), ak = a_kc ? ((e & 3) << 2) : (e >> 5);
                 const float4 v = __ldg(reinterpret_cast<const float4*>(d.A + (m0 + am) * d.a_sm + (k0 + ak) * d.a_sk));
                 ra[4 * i] = v.x; ra[4 * i + 1] = v.y; ra[4 * i + 2] = v.z; ra[4 * i + 3] = v.w;
+                if (TRANSFORM) {
+                    // the four logits run along the contiguous direction, which is the class: one pattern for all four
+                    const int64_t pat = d.a_pattern_is_m ? m0 + am : k0 + ak;
+                    const int64_t cls = d.a_pattern_is_m ? k0 + ak : m0 + am;
+                    const float l = __ldg(d.lse + pat);
+                    const int64_t lab = (int64_t)__ldg(d.labels + pat);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) ra[4 * i + j] = expf(ra[4 * i + j] - l) - (cls + j == lab ? 1.f : 0.f);
+                }
             }
         } else {
 #pragma unroll
