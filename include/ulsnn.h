@@ -178,6 +178,19 @@ ulsnn_status_t ulsnn_mlp_gradient_sse(ulsnn_mlp_t* handle, const float* const* W
 /* Section 4.2: W := W - lr * dW, b := b - lr * db, in place, one fused multiply-add per element. */
 ulsnn_status_t ulsnn_sgd_step(ulsnn_mlp_t* handle, float* const* W, float* const* b,
                               const float* const* dW, const float* const* db, float lr, ulsnn_stream_t stream);
+/*
+ * Vector operations for the line search and the conjugate-gradient direction of Section 4.2, on flat parameter
+ * vectors in device memory.
+ * ulsnn_vec_dot: *out (device, one double) = sum_i x[i]*y[i], accumulated in double in an order that depends on n
+ *   only (partial sums over blocks of 1024 elements, then a fixed tree), so repeated runs give the same bits.
+ *   workspace: device scratch of ulsnn_vec_dot_workspace_bytes(n) bytes, 8-byte aligned.
+ * ulsnn_vec_axpby: out[i] = a*x[i] + b*y[i]; out may be x or y.
+ */
+ulsnn_status_t ulsnn_vec_dot_workspace_bytes(int64_t n, size_t* bytes /* host, out */);
+ulsnn_status_t ulsnn_vec_dot(int64_t n, const float* x, const float* y, double* out, void* workspace,
+                             size_t workspace_bytes, ulsnn_stream_t stream);
+ulsnn_status_t ulsnn_vec_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out,
+                               ulsnn_stream_t stream);
 /* Synchronises `stream`, then returns ULSNN_OK, ULSNN_ERR_DEVICE_TIMEOUT if a kernel of this handle gave up a
  * bounded wait since the last call of this function (the word is cleared), or ULSNN_ERR_CUDA. */
 ulsnn_status_t ulsnn_last_device_status(ulsnn_mlp_t* handle, ulsnn_stream_t stream);

@@ -7,4 +7,4 @@ csrc/; `paper_1911_05181_b200.binding` is the thin ctypes layer over it.
 Importing this package does not load the library; `binding.lib()` does, and it
 raises if the library has not been built.
 """
-__all__ = ["binding", "flops", "buildlib", "dp"]
+__all__ = ["binding", "flops", "buildlib", "dp", "cg"]

@@ -31,6 +31,7 @@ EXPORTS = [
     "ulsnn_mlp_gradient", "ulsnn_sgd_step", "ulsnn_last_device_status", "ulsnn_fill_uniform",
     "ulsnn_fill_labels", "ulsnn_launch_counts", "ulsnn_mlp_enable_timing", "ulsnn_mlp_phase_times",
     "ulsnn_sgemm_noalloc", "ulsnn_sgemm_noalloc_max_scratch_bytes", "ulsnn_mlp_forward_sse", "ulsnn_mlp_gradient_sse",
+    "ulsnn_vec_dot_workspace_bytes", "ulsnn_vec_dot", "ulsnn_vec_axpby",
 ]
 
 
@@ -76,6 +77,9 @@ def lib():
         l.ulsnn_mlp_gradient.argtypes = [vp, pp, pp, vp, i64, vp, i64, ctypes.c_int, pp, pp, vp, vp]
         l.ulsnn_mlp_forward_sse.argtypes = [vp, pp, pp, vp, i64, vp, i64, i64, vp, vp]
         l.ulsnn_mlp_gradient_sse.argtypes = [vp, pp, pp, vp, i64, vp, i64, i64, ctypes.c_int, pp, pp, vp, vp]
+        l.ulsnn_vec_dot_workspace_bytes.argtypes = [i64, ctypes.POINTER(sz)]
+        l.ulsnn_vec_dot.argtypes = [i64, vp, vp, vp, vp, sz, vp]
+        l.ulsnn_vec_axpby.argtypes = [i64, f32, vp, f32, vp, vp, vp]
         l.ulsnn_sgd_step.argtypes = [vp, pp, pp, pp, pp, f32, vp]
         l.ulsnn_last_device_status.argtypes = [vp, vp]
         l.ulsnn_fill_uniform.argtypes = [vp, i64, u64, u64, u64, ctypes.c_int, vp]
@@ -165,6 +169,20 @@ def sgemm_noalloc(transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, 
     if check:
         _check(st, "ulsnn_sgemm_noalloc")
     return st
+
+
+def vec_dot_workspace_bytes(n) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().ulsnn_vec_dot_workspace_bytes(n, ctypes.byref(out)), "ulsnn_vec_dot_workspace_bytes")
+    return out.value
+
+
+def vec_dot(n, x, y, out, workspace, workspace_bytes, stream=None):
+    _check(lib().ulsnn_vec_dot(n, _ptr(x), _ptr(y), _ptr(out), _ptr(workspace), workspace_bytes, _stream(stream)), "ulsnn_vec_dot")
+
+
+def vec_axpby(n, a, x, b, y, out, stream=None):
+    _check(lib().ulsnn_vec_axpby(n, a, _ptr(x), b, _ptr(y), _ptr(out), _stream(stream)), "ulsnn_vec_axpby")
 
 
 def fill_uniform(dst, n, seed, tensor_id, offset=0, mode=0, stream=None):

@@ -694,6 +694,31 @@ extern "C" ulsnn_status_t ulsnn_sgd_step(ulsnn_mlp_t* h, float* const* W, float*
     return ULSNN_OK;
 }
 
+extern "C" ulsnn_status_t ulsnn_vec_dot_workspace_bytes(int64_t n, size_t* bytes) {
+    if (!bytes || n < 0) return ULSNN_ERR_INVALID_ARG;
+    *bytes = align256((size_t)(dot_parts(n) + 1) * sizeof(double));
+    return ULSNN_OK;
+}
+
+extern "C" ulsnn_status_t ulsnn_vec_dot(int64_t n, const float* x, const float* y, double* out, void* workspace,
+                                        size_t workspace_bytes, ulsnn_stream_t stream) {
+    if (n < 0 || !out || (n > 0 && (!x || !y))) return ULSNN_ERR_INVALID_ARG;
+    if (n > 0 && (!workspace || ((uintptr_t)workspace & 7) != 0)) return ULSNN_ERR_INVALID_ARG;
+    if ((size_t)(dot_parts(n) + 1) * sizeof(double) > workspace_bytes && n > 0) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
+    ulsnn_status_t st = check_arch();
+    if (st != ULSNN_OK) return st;
+    return launch_dot(n, x, y, out, (double*)workspace, (cudaStream_t)stream);
+}
+
+extern "C" ulsnn_status_t ulsnn_vec_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out,
+                                          ulsnn_stream_t stream) {
+    if (n < 0 || (n > 0 && (!x || !y || !out))) return ULSNN_ERR_INVALID_ARG;
+    if (n == 0) return ULSNN_OK;
+    ulsnn_status_t st = check_arch();
+    if (st != ULSNN_OK) return st;
+    return launch_axpby(n, a, x, b, y, out, (cudaStream_t)stream);
+}
+
 extern "C" ulsnn_status_t ulsnn_last_device_status(ulsnn_mlp_t* h, ulsnn_stream_t stream) {
     (void)h;
     int word = 0;

@@ -105,6 +105,10 @@ ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* lse
 int delta_colsum_tiles(int64_t n);
 // hi[i] = tf32_rn(x[i]), lo[i] = tf32_rn(x[i] - hi[i])   (round to nearest, ties away from zero, 10 mantissa bits)
 ulsnn_status_t launch_split_hilo(const float* x, int64_t n, float* hi, float* lo, cudaStream_t stream);
+// out = a*x + b*y (out may alias x or y); *out = sum_i x[i]*y[i] in double, blocks of 1024 elements in index order
+ulsnn_status_t launch_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out, cudaStream_t stream);
+ulsnn_status_t launch_dot(int64_t n, const float* x, const float* y, double* out, double* parts, cudaStream_t stream);
+int64_t dot_parts(int64_t n);
 ulsnn_status_t launch_sgd(float* w, const float* g, int64_t n, float lr, cudaStream_t stream);
 ulsnn_status_t launch_zero(float* p, int64_t n, cudaStream_t stream);
 ulsnn_status_t launch_zero_f64(double* p, int64_t n, cudaStream_t stream);

@@ -138,6 +138,44 @@ __global__ void split_hilo_kernel(const float* __restrict__ x, int64_t n, float*
     }
 }
 
+__global__ void axpby_kernel(int64_t n, float a, const float* __restrict__ x, float b, const float* __restrict__ y, float* out) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = fmaf(a, x[i], b * y[i]);
+}
+
+constexpr int DOT_BLOCK = 1024;     // elements per partial sum
+
+// partial sums of x*y over blocks of DOT_BLOCK elements: 256 threads take four elements each (index order inside a
+// thread), then a fixed tree over the threads; all in double
+__global__ void dot_parts_kernel(int64_t n, const float* __restrict__ x, const float* __restrict__ y, double* __restrict__ parts) {
+    __shared__ double red[256];
+    const int64_t base = (int64_t)blockIdx.x * DOT_BLOCK + (int64_t)threadIdx.x * 4;
+    double s = 0.0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) if (base + j < n) s += (double)x[base + j] * (double)y[base + j];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) parts[blockIdx.x] = red[0];
+}
+
+__global__ void dot_final_kernel(const double* __restrict__ parts, int64_t nparts, double* __restrict__ out) {
+    // one block: 256 threads add every 256th partial in index order, then a fixed tree
+    __shared__ double red[256];
+    double s = 0.0;
+    for (int64_t i = threadIdx.x; i < nparts; i += 256) s += parts[i];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = red[0];
+}
+
 __global__ void sgd_kernel(float* __restrict__ w, const float* __restrict__ g, int64_t n, float lr) {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         w[i] = fmaf(-lr, g[i], w[i]);
@@ -270,6 +308,28 @@ ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* lse
 ulsnn_status_t launch_split_hilo(const float* x, int64_t n, float* hi, float* lo, cudaStream_t stream) {
     if (n <= 0) return ULSNN_OK;
     split_hilo_kernel<<<grid_for(n, 256), 256, 0, stream>>>(x, n, hi, lo);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+ulsnn_status_t launch_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out, cudaStream_t stream) {
+    if (n <= 0) return ULSNN_OK;
+    axpby_kernel<<<grid_for(n, 256), 256, 0, stream>>>(n, a, x, b, y, out);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+int64_t dot_parts(int64_t n) { return n > 0 ? (n + DOT_BLOCK - 1) / DOT_BLOCK : 0; }
+
+ulsnn_status_t launch_dot(int64_t n, const float* x, const float* y, double* out, double* parts, cudaStream_t stream) {
+    const int64_t np = dot_parts(n);
+    if (np > 0x7fffffff) return ULSNN_ERR_TOO_LARGE;
+    if (np > 0) {
+        dot_parts_kernel<<<(unsigned)np, 256, 0, stream>>>(n, x, y, parts);
+        ulsnn::count_launch(2);
+        if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
+    }
+    dot_final_kernel<<<1, 256, 0, stream>>>(parts, np, out);
     ulsnn::count_launch(2);
     return cuda_ok(cudaGetLastError());
 }
