@@ -111,3 +111,34 @@ def test_fill_rejects_bad_arguments():
     assert lib.ulsnn_fill_uniform(4096, 4, 0, 0, 0, 5, None) == ul.ERR_INVALID_ARG
     assert lib.ulsnn_fill_labels(4096, 4, 0, 0, 0, 0, None) == ul.ERR_INVALID_ARG
     assert lib.ulsnn_fill_uniform(None, 0, 0, 0, 0, 0, None) == ul.OK
+
+
+def test_vector_calls_reject_bad_arguments_on_the_host():
+    fake = 4096
+    out = ctypes.c_size_t(0)
+    lib = ul.lib()
+    assert lib.ulsnn_vec_dot_workspace_bytes(-1, ctypes.byref(out)) == ul.ERR_INVALID_ARG
+    assert lib.ulsnn_vec_dot_workspace_bytes(5000, ctypes.byref(out)) == ul.OK and out.value >= 6 * 8
+    assert lib.ulsnn_vec_dot(10, fake, fake, None, fake, 4096, None) == ul.ERR_INVALID_ARG        # no output
+    assert lib.ulsnn_vec_dot(10, None, fake, fake, fake, 4096, None) == ul.ERR_INVALID_ARG
+    assert lib.ulsnn_vec_dot(5000, fake, fake, fake, fake, 8, None) == ul.ERR_WORKSPACE_TOO_SMALL
+    assert lib.ulsnn_vec_axpby(-3, 1.0, fake, 1.0, fake, fake, None) == ul.ERR_INVALID_ARG
+    assert lib.ulsnn_vec_axpby(0, 1.0, None, 1.0, None, None, None) == ul.OK
+
+
+def test_squared_error_head_rejects_bad_arguments_on_the_host():
+    sizes = [8, 4, 3]
+    nbytes = ul.mlp_workspace_bytes(sizes, ul.MATH_FP32_SIMT, 16)
+    arr = (ctypes.c_int32 * 3)(*sizes)
+    d = ul._Desc(2, arr, ul.MATH_FP32_SIMT, 16)
+    h = ctypes.c_void_p(None)
+    assert ul.lib().ulsnn_mlp_create(ctypes.byref(h), ctypes.byref(d), 4096, nbytes) == ul.OK     # 4096: aligned, never touched
+    fake = 8192
+    ptrs = (ctypes.c_void_p * 2)(fake, fake)
+    lib = ul.lib()
+    assert lib.ulsnn_mlp_forward_sse(h, ptrs, ptrs, fake, 8, None, 3, 4, fake, None) == ul.ERR_INVALID_ARG      # no targets
+    assert lib.ulsnn_mlp_forward_sse(h, ptrs, ptrs, fake, 8, fake, 2, 4, fake, None) == ul.ERR_INVALID_ARG      # ldt < classes
+    assert lib.ulsnn_mlp_forward_sse(h, ptrs, ptrs, fake, 7, fake, 3, 4, fake, None) == ul.ERR_INVALID_ARG      # ldx < inputs
+    assert lib.ulsnn_mlp_gradient_sse(h, ptrs, ptrs, fake, 8, fake, 3, 17, 0, ptrs, ptrs, fake, None) == ul.ERR_INVALID_ARG   # n > max
+    assert lib.ulsnn_mlp_gradient_sse(h, ptrs, ptrs, fake, 8, fake, 3, 4, 0, None, ptrs, fake, None) == ul.ERR_INVALID_ARG
+    lib.ulsnn_mlp_destroy(h)
