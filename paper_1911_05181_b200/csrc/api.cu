@@ -302,6 +302,7 @@ struct ulsnn_mlp {
     float* Zlo;                     // 3xTF32, squared-error head: lo half of the output deltas (Z holds the hi half)
     float2* stats;
     float* lse;
+    float* chunk_tab; int64_t chunk_ld;     // per pattern and 32-class chunk: chunk maximum, then the factor exp(m - lse)
     float* zlabel;
     double* loss_parts;
     float* colsum_parts;
@@ -365,6 +366,8 @@ ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
     h->stats_ld = ((int64_t)h->sizes[L] + 63) / 64;          // enough for any column-tile width >= 64
     h->stats = (float2*)take((size_t)B * h->stats_ld * sizeof(float2));
     h->lse = (float*)take((size_t)B * sizeof(float));
+    h->chunk_ld = round_up(((int64_t)h->sizes[L] + 31) / 32, 4);
+    h->chunk_tab = (float*)take((size_t)B * h->chunk_ld * sizeof(float));
     h->zlabel = (float*)take((size_t)B * sizeof(float));
     h->loss_parts = (double*)take((size_t)(rowstats_blocks(B) + 1) * sizeof(double));
     size_t cs = 0;
@@ -464,6 +467,7 @@ ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* 
         d.C_lo = keep_logits ? h->Zlo : nullptr;
     }
     d.stats = h->stats; d.stats_ld = h->stats_ld; d.zlabel = h->zlabel;
+    d.chunk_max = (keep_logits && !tg.T) ? h->chunk_tab : nullptr; d.chunk_ld = h->chunk_ld;
     d.splits = 1; d.k_per_split = d.K;
     const bool tc = use_tc(d, h->math);
     const int64_t bn = tc ? tc_tile_n(d) : simt_tile_n();
@@ -472,7 +476,8 @@ ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* 
     ulsnn_status_t st = timed_gemm(h, d, stream);
     if (st != ULSNN_OK) return st;
     if (tg.T) return launch_rowsums(h->stats, h->stats_ld, tiles, n, h->loss_parts, accumulate, loss_out, stream);
-    return launch_rowstats(h->stats, h->stats_ld, tiles, h->zlabel, n, h->lse, h->loss_parts, accumulate, loss_out, stream);
+    return launch_rowstats(h->stats, h->stats_ld, tiles, h->zlabel, n, h->lse, d.chunk_max, h->chunk_ld,
+                           (int)(((int64_t)h->sizes[L] + 31) / 32), h->loss_parts, accumulate, loss_out, stream);
 }
 
 ulsnn_status_t check_call(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
@@ -599,7 +604,7 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
         if (l + 1 == L && sse) {
             d.A = h->Z; d.A_lo = h->Zlo; d.a_sm = h->ldz;
         } else if (l + 1 == L) {
-            d.A = h->Z; d.a_sm = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 1;
+            d.A = h->Z; d.a_sm = h->ldz; d.a_transform = 1; d.scale = h->chunk_tab; d.scale_ld = h->chunk_ld; d.labels = labels; d.a_pattern_is_m = 1;
             d.delta_out = h->D2; d.delta_out_lo = h->D2lo;      // kept for the weight-gradient product below
         }
         else            { d.A = h->D[l + 1]; d.a_sm = h->ldd[l + 1]; }
@@ -623,7 +628,7 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
         d.M = h->sizes[w + 1]; d.N = h->sizes[w] + (w >= 1 ? 1 : 0); d.K = n;
         if (w + 1 == L && sse) { d.A = h->Z; d.A_lo = h->Zlo; d.a_sk = h->ldz; }
         else if (w + 1 == L && delta2_kept) { d.A = h->D2; d.A_lo = h->D2lo; d.a_sk = h->ldz; }
-        else if (w + 1 == L) { d.A = h->Z; d.a_sk = h->ldz; d.a_transform = 1; d.lse = h->lse; d.labels = labels; d.a_pattern_is_m = 0; }
+        else if (w + 1 == L) { d.A = h->Z; d.a_sk = h->ldz; d.a_transform = 1; d.scale = h->chunk_tab; d.scale_ld = h->chunk_ld; d.labels = labels; d.a_pattern_is_m = 0; }
         else            { d.A = h->D[w + 1]; d.a_sk = h->ldd[w + 1]; }
         d.a_sm = 1;
         if (w >= 1) { d.B = h->H[w]; d.B_lo = h->Hlo[w]; d.b_sk = h->ldh[w]; } else { d.B = X; d.b_sk = ldx; }
@@ -644,7 +649,7 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
     } else if (sse) {
         st = launch_matrix_colsum(h->Z, h->Zlo, h->ldz, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);
     } else {
-        st = launch_delta_colsum(h->Z, h->ldz, h->lse, labels, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);
+        st = launch_delta_colsum(h->Z, h->ldz, h->chunk_tab, h->chunk_ld, labels, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);
     }
     return st;
 }

@@ -11,7 +11,8 @@ namespace ulsnn {
 enum Epilogue : int {
     EPI_SGEMM     = 0,  // C = alpha*acc + beta*C                                   (Section 3.1)
     EPI_BIAS_TANH = 1,  // C = tanh(acc + bias[col]); optionally C[:, N] = 1         (Eq. 2 / H = tanh(X W^T))
-    EPI_LOGITS    = 2,  // z = acc + bias[col]; per-(row, column-tile) softmax statistics, z at the label
+    EPI_LOGITS    = 2,  // z = acc + bias[col]; per-(row, column-tile) softmax statistics, z at the label; stored: exp(z - m)
+                        // with m the running maximum of the row when its 32-column chunk was reached (chunk_max)
     EPI_TANHP     = 3,  // C = (1 - h*h) * acc, h = Hm[row][col]; per-row-tile column sums (H_D of Section 4.2)
     EPI_PARTIAL   = 4,  // split-K slice: raw accumulator into partials[slice]
     EPI_TANH_SSE  = 5   // the paper's output layer (Eqs. 1, 3): y = tanh(acc + bias); per-(row, column-tile) sums of
@@ -41,9 +42,11 @@ struct GemmDesc {
     const float* T; int64_t ldt;         // TANH_SSE: targets [M x N], rows ldt apart
     float2* stats; int64_t stats_ld;     // LOGITS: stats[row*stats_ld + col_tile] = (max, sum exp(z - max)); TANH_SSE: (0, sum (y-t)^2)
     float* zlabel;            // LOGITS: z[row][label[row]]
-    // A transform: the stored operand holds logits z; the product uses softmax(z) - onehot(label)
+    float* chunk_max; int64_t chunk_ld;  // LOGITS: chunk_max[row*chunk_ld + col/32] = the m that chunk's stored values refer to
+    // A transform: the stored operand holds e = exp(z - m) as left by the LOGITS epilogue; the product uses
+    // softmax(z) - onehot(label) = e * scale - onehot, scale[pattern*scale_ld + class/32] = exp(m - logsumexp)
     int a_transform;
-    const float* lse;         // [patterns] log-sum-exp of each pattern's logits
+    const float* scale; int64_t scale_ld;
     int a_pattern_is_m;       // 1: the M index of A is the pattern (K is the class); 0: K is the pattern
     // Optional copy of the transformed operand (tensor-core engine, a_pattern_is_m == 1 only): delta = softmax - onehot
     // is also written to delta_out (and, in 3xTF32 mode, as the pair tf32_rn(delta) -> delta_out, remainder ->
@@ -88,9 +91,11 @@ ulsnn_status_t launch_splitk_reduce(const float* parts, int splits, int64_t M, i
 ulsnn_status_t launch_colsum_reduce(const float* parts, int64_t tiles, int64_t N, int accumulate, float* out,
                                     cudaStream_t stream);
 // lse[p] from the per-tile statistics; loss = sum_p (lse[p] - zlabel[p]) in a fixed order, in double
+// chunk_tab (may be null): [n x chunk_ld] chunk maxima written by the LOGITS epilogue, turned in place into the
+// factors exp(m - lse) that the delta products multiply the stored exponentials with
 ulsnn_status_t launch_rowstats(const float2* stats, int64_t stats_ld, int tiles, const float* zlabel, int64_t n,
-                               float* lse, double* block_partials, int accumulate, double* loss_out,
-                               cudaStream_t stream);
+                               float* lse, float* chunk_tab, int64_t chunk_ld, int n_chunks, double* block_partials,
+                               int accumulate, double* loss_out, cudaStream_t stream);
 int rowstats_blocks(int64_t n);
 // loss = sum_p sum_t stats[p*stats_ld + t].y in a fixed order, in double (the squared-error head)
 ulsnn_status_t launch_rowsums(const float2* stats, int64_t stats_ld, int tiles, int64_t n, double* block_partials,
@@ -98,8 +103,9 @@ ulsnn_status_t launch_rowsums(const float2* stats, int64_t stats_ld, int tiles, 
 // out[j] = sum_p (A[p*lda + j] + A_lo[p*lda + j])  (A_lo may be null), rows added in a fixed order
 ulsnn_status_t launch_matrix_colsum(const float* A, const float* A_lo, int64_t lda, int64_t n, int64_t cols, float* parts,
                                     int accumulate, float* out, cudaStream_t stream);
-// db[j] = sum_p softmax(z_p)_j - [label_p == j]   (only for networks without a hidden layer)
-ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* lse, const int32_t* labels,
+// db[j] = sum_p softmax(z_p)_j - [label_p == j]   (only for networks without a hidden layer); Z holds the stored
+// exponentials, scale their per-chunk factors
+ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* scale, int64_t scale_ld, const int32_t* labels,
                                    int64_t n, int64_t n_classes, float* parts, int accumulate, float* out,
                                    cudaStream_t stream);
 int delta_colsum_tiles(int64_t n);

@@ -54,6 +54,7 @@ constexpr int RS_THREADS = 256;
 // then sum lse - z_label over the block in a fixed tree.
 __global__ void rowstats_kernel(const float2* __restrict__ stats, int64_t stats_ld, int tiles,
                                 const float* __restrict__ zlabel, int64_t n, float* __restrict__ lse,
+                                float* __restrict__ chunk_tab, int64_t chunk_ld, int n_chunks,
                                 double* __restrict__ block_partials) {
     __shared__ double red[RS_THREADS];
     const int64_t p = (int64_t)blockIdx.x * RS_THREADS + threadIdx.x;
@@ -68,6 +69,8 @@ __global__ void rowstats_kernel(const float2* __restrict__ stats, int64_t stats_
         }
         const double l = (double)mx + log(s);
         lse[p] = (float)l;
+        if (chunk_tab)
+            for (int t = 0; t < n_chunks; ++t) chunk_tab[p * chunk_ld + t] = (float)exp((double)chunk_tab[p * chunk_ld + t] - l);
         term = l - (double)zlabel[p];
     }
     red[threadIdx.x] = term;
@@ -115,14 +118,14 @@ __global__ void matrix_colsum_kernel(const float* __restrict__ A, const float* _
     parts[(int64_t)blockIdx.y * cols + j] = s;
 }
 
-__global__ void delta_colsum_kernel(const float* __restrict__ Z, int64_t ldz, const float* __restrict__ lse,
+__global__ void delta_colsum_kernel(const float* __restrict__ Z, int64_t ldz, const float* __restrict__ scale, int64_t scale_ld,
                                     const int32_t* __restrict__ labels, int64_t n, int64_t n_classes,
                                     float* __restrict__ parts) {
     const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n_classes) return;
     const int64_t p0 = (int64_t)blockIdx.y * DC_ROWS, p1 = min(n, p0 + DC_ROWS);
     float s = 0.f;
-    for (int64_t p = p0; p < p1; ++p) s += expf(Z[p * ldz + j] - lse[p]) - ((int64_t)labels[p] == j ? 1.f : 0.f);
+    for (int64_t p = p0; p < p1; ++p) s += Z[p * ldz + j] * scale[p * scale_ld + (j >> 5)] - ((int64_t)labels[p] == j ? 1.f : 0.f);
     parts[(int64_t)blockIdx.y * n_classes + j] = s;
 }
 
@@ -250,11 +253,11 @@ ulsnn_status_t launch_colsum_reduce(const float* parts, int64_t tiles, int64_t N
 int rowstats_blocks(int64_t n) { return (int)((n + RS_THREADS - 1) / RS_THREADS); }
 
 ulsnn_status_t launch_rowstats(const float2* stats, int64_t stats_ld, int tiles, const float* zlabel, int64_t n,
-                               float* lse, double* block_partials, int accumulate, double* loss_out,
-                               cudaStream_t stream) {
+                               float* lse, float* chunk_tab, int64_t chunk_ld, int n_chunks, double* block_partials,
+                               int accumulate, double* loss_out, cudaStream_t stream) {
     const int nb = rowstats_blocks(n);
     if (nb > 0) {
-        rowstats_kernel<<<nb, RS_THREADS, 0, stream>>>(stats, stats_ld, tiles, zlabel, n, lse, block_partials);
+        rowstats_kernel<<<nb, RS_THREADS, 0, stream>>>(stats, stats_ld, tiles, zlabel, n, lse, chunk_tab, chunk_ld, n_chunks, block_partials);
         ulsnn::count_launch(2);
         if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
     }
@@ -291,14 +294,14 @@ ulsnn_status_t launch_matrix_colsum(const float* A, const float* A_lo, int64_t l
 
 int delta_colsum_tiles(int64_t n) { return (int)((n + DC_ROWS - 1) / DC_ROWS); }
 
-ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* lse, const int32_t* labels,
+ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* scale, int64_t scale_ld, const int32_t* labels,
                                    int64_t n, int64_t n_classes, float* parts, int accumulate, float* out,
                                    cudaStream_t stream) {
     const int tiles = delta_colsum_tiles(n);
     if (tiles > 65535) return ULSNN_ERR_TOO_LARGE;
     if (tiles > 0) {
         dim3 grid((unsigned)((n_classes + 127) / 128), (unsigned)tiles);
-        delta_colsum_kernel<<<grid, 128, 0, stream>>>(Z, ldz, lse, labels, n, n_classes, parts);
+        delta_colsum_kernel<<<grid, 128, 0, stream>>>(Z, ldz, scale, scale_ld, labels, n, n_classes, parts);
         ulsnn::count_launch(2);
         if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
     }

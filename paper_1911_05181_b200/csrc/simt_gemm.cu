@@ -23,7 +23,7 @@ __device__ __forceinline__ float load_a(const GemmDesc& d, int64_t i, int64_t k,
     if (TRANSFORM) {
         const int64_t p = d.a_pattern_is_m ? i : k;
         const int64_t c = d.a_pattern_is_m ? k : i;
-        z = expf(z - __ldg(d.lse + p)) - ((int64_t)__ldg(d.labels + p) == c ? 1.f : 0.f);
+        z = z * __ldg(d.scale + p * d.scale_ld + (c >> 5)) - ((int64_t)__ldg(d.labels + p) == c ? 1.f : 0.f);
     }
     return z;
 }
@@ -70,13 +70,14 @@ __global__ void __launch_bounds__(NT, 2) simt_gemm_kernel(const GemmDesc d) {
                 const float4 v = __ldg(reinterpret_cast<const float4*>(d.A + (m0 + am) * d.a_sm + (k0 + ak) * d.a_sk));
                 ra[4 * i] = v.x; ra[4 * i + 1] = v.y; ra[4 * i + 2] = v.z; ra[4 * i + 3] = v.w;
                 if (TRANSFORM) {
-                    // the four logits run along the contiguous direction, which is the class: one pattern for all four
+                    // the four values run along the contiguous direction, which is the class: one pattern and one
+                    // 32-class chunk (cls is a multiple of 4) for all four
                     const int64_t pat = d.a_pattern_is_m ? m0 + am : k0 + ak;
                     const int64_t cls = d.a_pattern_is_m ? k0 + ak : m0 + am;
-                    const float l = __ldg(d.lse + pat);
+                    const float sc = __ldg(d.scale + pat * d.scale_ld + (cls >> 5));
                     const int64_t lab = (int64_t)__ldg(d.labels + pat);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) ra[4 * i + j] = expf(ra[4 * i + j] - l) - (cls + j == lab ? 1.f : 0.f);
+                    for (int j = 0; j < 4; ++j) ra[4 * i + j] = ra[4 * i + j] * sc - (cls + j == lab ? 1.f : 0.f);
                 }
             }
         } else {
@@ -243,19 +244,25 @@ __global__ void __launch_bounds__(NT, 2) simt_gemm_kernel(const GemmDesc d) {
             }
 #pragma unroll
             for (int o = 8; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            float s = 0.f;
+            float s = 0.f, e[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) s += (v[j] == -INFINITY) ? 0.f : expf(v[j] - mx);
+            for (int j = 0; j < 8; ++j) { e[j] = (v[j] == -INFINITY) ? 0.f : expf(v[j] - mx); s += e[j]; }
 #pragma unroll
             for (int o = 8; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             if (rv) {
-                if (tx == 0) d.stats[r * d.stats_ld + blockIdx.y] = make_float2(mx, s);
+                if (tx == 0) {
+                    d.stats[r * d.stats_ld + blockIdx.y] = make_float2(mx, s);
+                    // the stored exponentials of this tile's four 32-column chunks all refer to the tile maximum
+                    if (d.chunk_max)
+                        for (int q = 0; q < BN / 32; ++q)
+                            if (n0 + 32 * q < d.N) d.chunk_max[r * d.chunk_ld + (n0 >> 5) + q] = mx;
+                }
                 const int64_t lab = (int64_t)__ldg(d.labels + r);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const int64_t c = col_of(j);
                     if (c < d.N) {
-                        if (d.C) d.C[r * d.ldc + c] = v[j];
+                        if (d.C) d.C[r * d.ldc + c] = e[j];
                         if (c == lab) d.zlabel[r] = v[j];
                     }
                 }

@@ -350,11 +350,9 @@ __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
     return v[0];
 }
 
-// softmax(z) - onehot from a stored logit: e = exp(z - lse) - [cls == label], 0 outside the matrix
-template <bool FAST>
-__device__ __forceinline__ float delta_of(float z, float lse, int cls, int label, int n_classes) {
-    const float e = exp_t<FAST>(z - lse) - (cls == label ? 1.f : 0.f);
-    return cls < n_classes ? e : 0.f;
+// softmax(z) - onehot from a stored exponential e = exp(z - m) and its chunk's factor exp(m - lse); 0 outside the matrix
+__device__ __forceinline__ float delta_of(float e, float scale, int cls, int label, int n_classes) {
+    return cls < n_classes ? fmaf(e, scale, cls == label ? -1.f : 0.f) : 0.f;
 }
 
 // hi = tf32_rn(x), lo = tf32_rn(x - hi).  (The tensor core ignores the low 13 mantissa bits of a stored word, so the
@@ -739,25 +737,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                         for (int j = 0; j < 32; ++j) { if (j >= nvalid) v[j] = -INFINITY; cm = fmaxf(cm, v[j]); }
                         const float nm = fmaxf(run_m, cm);
-                        float s = 0.f;
-                        auto sum_exp = [&](auto fast_tag) {
-                            constexpr bool FAST = decltype(fast_tag)::value;
-                            if (full) {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) s += exp_t<FAST>(v[j] - nm);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) if (j < nvalid) s += exp_t<FAST>(v[j] - nm);
-                            }
-                            run_s = (run_m == -INFINITY ? 0.f : run_s * exp_t<FAST>(run_m - nm)) + s;
-                        };
-                        if (p.fast_math) sum_exp(std::true_type{}); else sum_exp(std::false_type{});
-                        run_m = nm;
                         if ((unsigned)(lab - c0) < (unsigned)nvalid) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (c0 + j == lab) zl = v[j];
                             have_zl = true;
                         }
+                        // the exponentials that make up the row sum are also what is stored: exp(z - nm), with nm
+                        // noted per chunk, so that the delta products get softmax(z) by one multiplication
+                        float s = 0.f;
+                        auto sum_exp = [&](auto fast_tag) {
+                            constexpr bool FAST = decltype(fast_tag)::value;
+                            if (full) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) { v[j] = exp_t<FAST>(v[j] - nm); s += v[j]; }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) { v[j] = (j < nvalid) ? exp_t<FAST>(v[j] - nm) : 0.f; s += v[j]; }
+                            }
+                            run_s = (run_m == -INFINITY ? 0.f : run_s * exp_t<FAST>(run_m - nm)) + s;
+                        };
+                        if (p.fast_math) sum_exp(std::true_type{}); else sum_exp(std::false_type{});
+                        run_m = nm;
+                        if (rv && d.chunk_max) d.chunk_max[r * d.chunk_ld + (c0 >> 5)] = nm;
                         do_store = d.C != nullptr;
                     }
                 } else if (EPI == EPI_TANHP) {
@@ -880,24 +881,44 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int b_cols = tile_cols(p, nt) / CG;
             // K-major logits (the pattern is the row): statistics of this thread's rows, once per tile
             constexpr int NA = (BM * BK / 4) / NT;          // 16-byte pieces of the A tile per thread
-            float row_lse[NA];
             int row_lab[NA];
 #pragma unroll
-            for (int i = 0; i < NA; ++i) { row_lse[i] = 0.f; row_lab[i] = -1; }
+            for (int i = 0; i < NA; ++i) row_lab[i] = -1;
             if (d.a_transform && !p.a_mn) {
 #pragma unroll
                 for (int i = 0; i < NA; ++i) {
                     const int pat = m0 + a_row + ROW_STEP * i;
-                    if (pat < n_patterns) { row_lse[i] = __ldg(d.lse + pat); row_lab[i] = __ldg(d.labels + pat); }
+                    if (pat < n_patterns) row_lab[i] = __ldg(d.labels + pat);
                 }
             }
             int k0 = (int)kbeg;
             for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
                 const int s = rp.stage;
                 // MN-major logits (the pattern is the k row): statistics of this thread's pattern in this block
-                float k_lse = 0.f; int k_lab = -1;
+                int k_lab = -1;
                 const int kpat = k0 + mn_krow;
-                if (d.a_transform && p.a_mn && kpat < n_patterns) { k_lse = __ldg(d.lse + kpat); k_lab = __ldg(d.labels + kpat); }
+                // factors of the 32-class chunks this thread's pieces lie in (fetched before the wait for the stage):
+                // K-major: the stage is one chunk (k0 is a multiple of 32) of each of the thread's rows;
+                // MN-major: the thread's pattern is fixed and its pieces lie in consecutive chunks
+                float pc_scale[NA];
+#pragma unroll
+                for (int i = 0; i < NA; ++i) pc_scale[i] = 0.f;
+                if (d.a_transform) {
+                    if (!p.a_mn) {
+#pragma unroll
+                        for (int i = 0; i < NA; ++i) {
+                            const int pat = m0 + a_row + ROW_STEP * i;
+                            if (pat < n_patterns && k0 < n_classes) pc_scale[i] = __ldg(d.scale + (int64_t)pat * d.scale_ld + (k0 >> 5));
+                        }
+                    } else if (kpat < n_patterns) {
+                        k_lab = __ldg(d.labels + kpat);
+#pragma unroll
+                        for (int i = 0; i < NA; ++i) {
+                            const int cls0 = m0 + 32 * (mn_g0 + mn_gstep * i);
+                            if (cls0 < n_classes) pc_scale[i] = __ldg(d.scale + (int64_t)kpat * d.scale_ld + (cls0 >> 5));
+                        }
+                    }
+                }
                 if (!wait_bar(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
                 rp.advance(p.stages);
                 uint8_t* base = stage_base + (size_t)s * p.stage_bytes;
@@ -905,9 +926,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 float4* a_lo = reinterpret_cast<float4*>(base + off_a_lo);
                 float4* b_hi = reinterpret_cast<float4*>(base + off_b_hi);
                 float4* b_lo = reinterpret_cast<float4*>(base + off_b_lo);
-                // The body is instantiated per (approximate exp?, 3xTF32?) so that its unrolled loops are straight-line code.
-                auto pass = [&](auto fast_tag, auto three_tag) {
-                    constexpr bool FAST = decltype(fast_tag)::value, THREE = decltype(three_tag)::value;
+                // The body is instantiated per mode so that its unrolled loops are straight-line code.
+                auto pass = [&](auto three_tag) {
+                    constexpr bool THREE = decltype(three_tag)::value;
                     if (!p.a_pre) {
                     float4 x[NA];
 #pragma unroll
@@ -918,20 +939,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                             for (int i = 0; i < NA; ++i) {
                                 const bool live = m0 + a_row + ROW_STEP * i < n_patterns;
-                                x[i].x = live ? delta_of<FAST>(x[i].x, row_lse[i], cls + 0, row_lab[i], n_classes) : 0.f;
-                                x[i].y = live ? delta_of<FAST>(x[i].y, row_lse[i], cls + 1, row_lab[i], n_classes) : 0.f;
-                                x[i].z = live ? delta_of<FAST>(x[i].z, row_lse[i], cls + 2, row_lab[i], n_classes) : 0.f;
-                                x[i].w = live ? delta_of<FAST>(x[i].w, row_lse[i], cls + 3, row_lab[i], n_classes) : 0.f;
+                                x[i].x = live ? delta_of(x[i].x, pc_scale[i], cls + 0, row_lab[i], n_classes) : 0.f;
+                                x[i].y = live ? delta_of(x[i].y, pc_scale[i], cls + 1, row_lab[i], n_classes) : 0.f;
+                                x[i].z = live ? delta_of(x[i].z, pc_scale[i], cls + 2, row_lab[i], n_classes) : 0.f;
+                                x[i].w = live ? delta_of(x[i].w, pc_scale[i], cls + 3, row_lab[i], n_classes) : 0.f;
                             }
                         } else {
                             const bool live = kpat < n_patterns;
 #pragma unroll
                             for (int i = 0; i < NA; ++i) {
                                 const int cls = m0 + 32 * (mn_g0 + mn_gstep * i) + mch * 4;
-                                x[i].x = live ? delta_of<FAST>(x[i].x, k_lse, cls + 0, k_lab, n_classes) : 0.f;
-                                x[i].y = live ? delta_of<FAST>(x[i].y, k_lse, cls + 1, k_lab, n_classes) : 0.f;
-                                x[i].z = live ? delta_of<FAST>(x[i].z, k_lse, cls + 2, k_lab, n_classes) : 0.f;
-                                x[i].w = live ? delta_of<FAST>(x[i].w, k_lse, cls + 3, k_lab, n_classes) : 0.f;
+                                x[i].x = live ? delta_of(x[i].x, pc_scale[i], cls + 0, k_lab, n_classes) : 0.f;
+                                x[i].y = live ? delta_of(x[i].y, pc_scale[i], cls + 1, k_lab, n_classes) : 0.f;
+                                x[i].z = live ? delta_of(x[i].z, pc_scale[i], cls + 2, k_lab, n_classes) : 0.f;
+                                x[i].w = live ? delta_of(x[i].w, pc_scale[i], cls + 3, k_lab, n_classes) : 0.f;
                             }
                         }
                     }
@@ -954,9 +975,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                     }
                 };
-                if (p.three_x) pass(std::false_type{}, std::true_type{});
-                else if (p.fast_math) pass(std::true_type{}, std::false_type{});
-                else pass(std::false_type{}, std::false_type{});
+                if (p.three_x) pass(std::true_type{}); else pass(std::false_type{});
                 proxy_fence_async();            // make these generic-proxy writes visible to the tensor core's reads
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->ready[s]));
