@@ -366,7 +366,7 @@ ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
     h->stats_ld = ((int64_t)h->sizes[L] + 63) / 64;          // enough for any column-tile width >= 64
     h->stats = (float2*)take((size_t)B * h->stats_ld * sizeof(float2));
     h->lse = (float*)take((size_t)B * sizeof(float));
-    h->chunk_ld = round_up(((int64_t)h->sizes[L] + 31) / 32, 4);
+    h->chunk_ld = round_up(((int64_t)h->sizes[L] + 31) / 32, 8);      // whole 256-column tiles: the epilogue writes eight at a time
     h->chunk_tab = (float*)take((size_t)B * h->chunk_ld * sizeof(float));
     h->zlabel = (float*)take((size_t)B * sizeof(float));
     h->loss_parts = (double*)take((size_t)(rowstats_blocks(B) + 1) * sizeof(double));

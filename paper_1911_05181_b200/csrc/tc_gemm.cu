@@ -654,6 +654,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int64_t r = (int64_t)r0w + lane;
             const bool rv = r < d.M;
             float run_m = -INFINITY, run_s = 0.f, zl = 0.f;
+            float tile_max[BN_MAX / 32];            // LOGITS: the maximum each chunk's stored exponentials refer to
+#pragma unroll
+            for (int c = 0; c < BN_MAX / 32; ++c) tile_max[c] = 0.f;
             int lab = -1;
             bool have_zl = false;
             if (EPI == EPI_LOGITS && rv) lab = __ldg(d.labels + r);
@@ -758,7 +761,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         };
                         if (p.fast_math) sum_exp(std::true_type{}); else sum_exp(std::false_type{});
                         run_m = nm;
-                        if (rv && d.chunk_max) d.chunk_max[r * d.chunk_ld + (c0 >> 5)] = nm;
+#pragma unroll
+                        for (int q8 = 0; q8 < BN_MAX / 32; ++q8) if (q8 == c) tile_max[q8] = nm;      // static indices: stays in registers
                         do_store = d.C != nullptr;
                     }
                 } else if (EPI == EPI_TANHP) {
@@ -842,6 +846,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (lane == 0) { if (CG == 2 && rank == 1) signal_rank0(smem_u32(&ctrl->free_sink[acc][ew]), smem_u32(&ctrl->reg_free[acc])); else mbar_arrive(smem_u32(&ctrl->reg_free[acc])); }
 
             if (EPI == EPI_TANH_SSE && rv) d.stats[r * d.stats_ld + nt] = make_float2(0.f, run_s);
+            if (EPI == EPI_LOGITS && rv && d.chunk_max) {
+                // the tile's chunk maxima in one go: the table's rows are padded to whole tiles
+                float4* dst = reinterpret_cast<float4*>(d.chunk_max + r * d.chunk_ld + (n0 >> 5));
+                dst[0] = make_float4(tile_max[0], tile_max[1], tile_max[2], tile_max[3]);
+                dst[1] = make_float4(tile_max[4], tile_max[5], tile_max[6], tile_max[7]);
+            }
             if (EPI == EPI_LOGITS && rv) {
                 d.stats[r * d.stats_ld + nt] = make_float2(run_m, run_s);
                 if (have_zl) d.zlabel[r] = zl;
