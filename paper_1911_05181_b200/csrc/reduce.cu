@@ -50,32 +50,47 @@ colsum_reduce_kernel(const float* __restrict__ parts, int64_t tiles, int64_t N, 
 
 constexpr int RS_THREADS = 256;
 
-// One thread per pattern: combine the per-tile (max, sum-exp) pairs in tile order into the log-sum-exp,
-// then sum lse - z_label over the block in a fixed tree.
-__global__ void rowstats_kernel(const float2* __restrict__ stats, int64_t stats_ld, int tiles,
-                                const float* __restrict__ zlabel, int64_t n, float* __restrict__ lse,
-                                float* __restrict__ chunk_tab, int64_t chunk_ld, int n_chunks,
-                                double* __restrict__ block_partials) {
-    __shared__ double red[RS_THREADS];
-    const int64_t p = (int64_t)blockIdx.x * RS_THREADS + threadIdx.x;
-    double term = 0.0;
-    if (p < n) {
-        float mx = -INFINITY;
-        for (int t = 0; t < tiles; ++t) mx = fmaxf(mx, stats[p * stats_ld + t].x);
-        double s = 0.0;
-        for (int t = 0; t < tiles; ++t) {
-            const float2 v = stats[p * stats_ld + t];
-            s += (double)v.y * exp((double)v.x - (double)mx);
+// One warp per pattern (each of a block's 8 warps takes 8 patterns in turn): the lanes combine the per-tile
+// (max, sum-exp) pairs -- every lane its tiles in index order, then a fixed shuffle tree -- into the log-sum-exp,
+// and turn the pattern's chunk maxima into the factors exp(m - lse).  lse - z_label is then summed over the
+// block's 64 patterns in a fixed tree.
+constexpr int RS_ROWS = 64;
+__global__ void __launch_bounds__(RS_THREADS)
+rowstats_kernel(const float2* __restrict__ stats, int64_t stats_ld, int tiles,
+                const float* __restrict__ zlabel, int64_t n, float* __restrict__ lse,
+                float* __restrict__ chunk_tab, int64_t chunk_ld, int n_chunks,
+                double* __restrict__ block_partials) {
+    __shared__ double red[RS_ROWS];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = 0; i < RS_ROWS / 8; ++i) {
+        const int row = warp * (RS_ROWS / 8) + i;
+        const int64_t p = (int64_t)blockIdx.x * RS_ROWS + row;
+        double term = 0.0;
+        if (p < n) {                                        // uniform over the warp
+            const float2* st = stats + p * stats_ld;
+            float mx = -INFINITY;
+            for (int t = lane; t < tiles; t += 32) mx = fmaxf(mx, st[t].x);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            double s = 0.0;
+            for (int t = lane; t < tiles; t += 32) {
+                const float2 v = st[t];
+                s += (double)v.y * exp((double)v.x - (double)mx);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            const double l = (double)mx + log(s);
+            if (chunk_tab) {
+                float* q = chunk_tab + p * chunk_ld;
+                for (int t = lane; t < n_chunks; t += 32) q[t] = expf((float)((double)q[t] - l));
+            }
+            if (lane == 0) lse[p] = (float)l;
+            term = l - (double)zlabel[p];
         }
-        const double l = (double)mx + log(s);
-        lse[p] = (float)l;
-        if (chunk_tab)
-            for (int t = 0; t < n_chunks; ++t) chunk_tab[p * chunk_ld + t] = (float)exp((double)chunk_tab[p * chunk_ld + t] - l);
-        term = l - (double)zlabel[p];
+        if (lane == 0) red[row] = term;
     }
-    red[threadIdx.x] = term;
     __syncthreads();
-    for (int o = RS_THREADS / 2; o > 0; o >>= 1) {
+    for (int o = RS_ROWS / 2; o > 0; o >>= 1) {
         if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
         __syncthreads();
     }
@@ -250,7 +265,7 @@ ulsnn_status_t launch_colsum_reduce(const float* parts, int64_t tiles, int64_t N
     return cuda_ok(cudaGetLastError());
 }
 
-int rowstats_blocks(int64_t n) { return (int)((n + RS_THREADS - 1) / RS_THREADS); }
+int rowstats_blocks(int64_t n) { return (int)((n + RS_ROWS - 1) / RS_ROWS); }
 
 ulsnn_status_t launch_rowstats(const float2* stats, int64_t stats_ld, int tiles, const float* zlabel, int64_t n,
                                float* lse, float* chunk_tab, int64_t chunk_ld, int n_chunks, double* block_partials,
@@ -268,7 +283,7 @@ ulsnn_status_t launch_rowstats(const float2* stats, int64_t stats_ld, int tiles,
 
 ulsnn_status_t launch_rowsums(const float2* stats, int64_t stats_ld, int tiles, int64_t n, double* block_partials,
                               int accumulate, double* loss_out, cudaStream_t stream) {
-    const int nb = rowstats_blocks(n);
+    const int nb = (int)((n + RS_THREADS - 1) / RS_THREADS);        // never more than rowstats_blocks(n): the buffer fits
     if (nb > 0) {
         rowsums_kernel<<<nb, RS_THREADS, 0, stream>>>(stats, stats_ld, tiles, n, block_partials);
         ulsnn::count_launch(2);
