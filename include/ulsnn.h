@@ -45,7 +45,10 @@ typedef int ulsnn_status_t;
 typedef enum {
     ULSNN_MATH_3XTF32    = 0,  /* tensor cores, each operand split hi+lo in TF32, three products: fp32-level accuracy */
     ULSNN_MATH_TF32      = 1,  /* tensor cores, operands truncated to TF32 (10-bit mantissa): fast mode */
-    ULSNN_MATH_FP32_SIMT = 2   /* FFMA on the CUDA cores: exact fp32 products, the comparison kernel */
+    ULSNN_MATH_FP32_SIMT = 2,  /* FFMA on the CUDA cores: exact fp32 products, the comparison kernel */
+    ULSNN_MATH_BF16      = 3   /* tensor cores, operands and stored activations / deltas rounded to bfloat16 (8-bit
+                                  mantissa), hardware tanh and exp approximations: the 16-bit mode (Section 1: 16 bits
+                                  are enough for smaller networks), twice the tensor rate and half the bytes of TF32 */
 } ulsnn_math_t;
 
 /* A CUDA stream (cudaStream_t / CUstream); 0 is the legacy default stream. */

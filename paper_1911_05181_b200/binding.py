@@ -23,7 +23,8 @@ ERR_TOO_LARGE = -6
 MATH_3XTF32 = 0
 MATH_TF32 = 1
 MATH_FP32_SIMT = 2
-MATH_NAMES = {MATH_3XTF32: "3xtf32", MATH_TF32: "tf32", MATH_FP32_SIMT: "fp32_simt"}
+MATH_BF16 = 3
+MATH_NAMES = {MATH_3XTF32: "3xtf32", MATH_TF32: "tf32", MATH_FP32_SIMT: "fp32_simt", MATH_BF16: "bf16"}
 
 EXPORTS = [
     "ulsnn_status_string", "ulsnn_version", "ulsnn_sgemm", "ulsnn_sgemm_ex", "ulsnn_sgemm_workspace_bytes",

@@ -55,7 +55,7 @@ struct SplitPlan { int splits; int64_t k_per_split; };
 
 // Fixed by the shapes only.  Slices are at most SLICE_CAP long once K is large (bounds the fp32 rounding of a
 // long sum), and short-and-wide products get enough slices to fill the GPU.
-SplitPlan plan_splits(int64_t tiles, int64_t K, int64_t slots) {
+SplitPlan plan_splits(int64_t tiles, int64_t K, int64_t slots, int64_t granule = 32) {
     int64_t s_acc = (K > 2 * SLICE_CAP) ? (K + SLICE_CAP - 1) / SLICE_CAP : 1;
     int64_t s_fill = 1;
     if (tiles < slots && K >= 1024) {
@@ -64,8 +64,8 @@ SplitPlan plan_splits(int64_t tiles, int64_t K, int64_t slots) {
         if (s_fill < 1) s_fill = 1;
     }
     int64_t s = s_acc > s_fill ? s_acc : s_fill;
-    int64_t kps = round_up((K + s - 1) / s, 32);
-    if (kps < 32) kps = 32;
+    int64_t kps = round_up((K + s - 1) / s, granule);
+    if (kps < granule) kps = granule;
     s = (K + kps - 1) / kps;
     if (s < 1) s = 1;
     return SplitPlan{(int)s, kps};
@@ -111,6 +111,8 @@ size_t sgemm_ws_for(const GemmDesc& d, bool tc) {
     return align256((size_t)p.splits * (size_t)d.M * (size_t)round_up(d.N, 4) * sizeof(float));
 }
 
+ulsnn_status_t half_sgemm_impl(const SgemmArgs& a, void* ws, size_t ws_bytes, cudaStream_t stream);
+
 ulsnn_status_t sgemm_impl(const SgemmArgs& a, ulsnn_math_t math, void* ws, size_t ws_bytes, cudaStream_t stream) {
     if (a.M == 0 || a.N == 0) return ULSNN_OK;
     if (!a.C) return ULSNN_ERR_INVALID_ARG;
@@ -119,6 +121,7 @@ ulsnn_status_t sgemm_impl(const SgemmArgs& a, ulsnn_math_t math, void* ws, size_
         return launch_scale_rows(a.C, a.M, a.N, a.ldc, a.beta, stream);
     }
     if (!a.A || !a.B) return ULSNN_ERR_INVALID_ARG;
+    if (math == ULSNN_MATH_BF16) return half_sgemm_impl(a, ws, ws_bytes, stream);
     GemmDesc d = sgemm_desc(a);
     const bool tc = use_tc(d, math);
     const SplitPlan p = plan_splits(tiles_of(d, tc), d.K, slots_of(d, tc));
@@ -132,6 +135,63 @@ ulsnn_status_t sgemm_impl(const SgemmArgs& a, ulsnn_math_t math, void* ws, size_
     ulsnn_status_t st = run_gemm(d, math, stream);
     if (st != ULSNN_OK) return st;
     return launch_splitk_reduce(d.partials, p.splits, d.M, d.N, ldp, a.alpha, a.beta, a.C, a.ldc, nullptr, stream);
+}
+
+// 16-bit mode: the operands are first rounded to bfloat16 into the workspace (rows padded to 8 elements), which
+// therefore holds [A as bf16][B as bf16][split-K partials].
+struct HalfSgemmPlan {
+    int64_t a_rows, a_cols, lda, b_rows, b_cols, ldb;
+    size_t a_bytes, b_bytes, part_bytes;
+    SplitPlan sp; int64_t ldp;
+};
+
+HalfGemmDesc half_sgemm_desc(const SgemmArgs& a, const HalfSgemmPlan& pl, const __nv_bfloat16* Ab, const __nv_bfloat16* Bb) {
+    HalfGemmDesc d{};
+    d.M = a.M; d.N = a.N; d.K = a.K;
+    d.A = Ab; d.a_sm = a.ta ? 1 : pl.lda; d.a_sk = a.ta ? pl.lda : 1;
+    d.B = Bb; d.b_sk = a.tb ? 1 : pl.ldb; d.b_sn = a.tb ? pl.ldb : 1;
+    d.C = a.C; d.ldc = a.ldc; d.alpha = a.alpha; d.beta = a.beta;
+    d.epi = EPI_SGEMM; d.splits = 1; d.k_per_split = a.K;
+    return d;
+}
+
+HalfSgemmPlan half_sgemm_plan(const SgemmArgs& a) {
+    HalfSgemmPlan pl{};
+    pl.a_rows = a.ta ? a.K : a.M; pl.a_cols = a.ta ? a.M : a.K; pl.lda = round_up(pl.a_cols, 8);
+    pl.b_rows = a.tb ? a.N : a.K; pl.b_cols = a.tb ? a.K : a.N; pl.ldb = round_up(pl.b_cols, 8);
+    pl.a_bytes = align256((size_t)pl.a_rows * pl.lda * 2);
+    pl.b_bytes = align256((size_t)pl.b_rows * pl.ldb * 2);
+    const HalfGemmDesc d = half_sgemm_desc(a, pl, nullptr, nullptr);
+    const int64_t tiles = ((d.M + hg_tile_m(d) - 1) / hg_tile_m(d)) * ((d.N + hg_tile_n(d) - 1) / hg_tile_n(d));
+    pl.sp = plan_splits(tiles, d.K, hg_slots(d), hg_k_granule());
+    pl.ldp = round_up(d.N, 4);
+    pl.part_bytes = pl.sp.splits <= 1 ? 0 : align256((size_t)pl.sp.splits * (size_t)d.M * (size_t)pl.ldp * sizeof(float));
+    return pl;
+}
+
+ulsnn_status_t half_sgemm_impl(const SgemmArgs& a, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    const HalfSgemmPlan pl = half_sgemm_plan(a);
+    const size_t need = pl.a_bytes + pl.b_bytes + pl.part_bytes;
+    if (!ws || ws_bytes < need) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
+    if (((uintptr_t)ws & 255) != 0) return ULSNN_ERR_INVALID_ARG;
+    __nv_bfloat16* Ab = (__nv_bfloat16*)ws;
+    __nv_bfloat16* Bb = (__nv_bfloat16*)((char*)ws + pl.a_bytes);
+    ulsnn_status_t st = launch_to_bf16(a.A, pl.a_rows, pl.a_cols, a.lda, Ab, pl.lda, 0, stream);
+    if (st != ULSNN_OK) return st;
+    if ((st = launch_to_bf16(a.B, pl.b_rows, pl.b_cols, a.ldb, Bb, pl.ldb, 0, stream)) != ULSNN_OK) return st;
+    HalfGemmDesc d = half_sgemm_desc(a, pl, Ab, Bb);
+    if (pl.sp.splits <= 1) return hg_gemm_launch(d, stream);
+    d.epi = EPI_PARTIAL; d.splits = pl.sp.splits; d.k_per_split = pl.sp.k_per_split;
+    d.partials = (float*)((char*)ws + pl.a_bytes + pl.b_bytes); d.ldp = pl.ldp;
+    if ((st = hg_gemm_launch(d, stream)) != ULSNN_OK) return st;
+    return launch_splitk_reduce(d.partials, pl.sp.splits, d.M, d.N, pl.ldp, a.alpha, a.beta, a.C, a.ldc, nullptr, stream);
+}
+
+// scratch a product needs in `math` (operands as given)
+size_t sgemm_need(const SgemmArgs& a, ulsnn_math_t math) {
+    if (math == ULSNN_MATH_BF16) { const HalfSgemmPlan pl = half_sgemm_plan(a); return pl.a_bytes + pl.b_bytes + pl.part_bytes; }
+    const GemmDesc d = sgemm_desc(a);
+    return sgemm_ws_for(d, use_tc(d, math));
 }
 
 // grow-only scratch of ulsnn_sgemm, one per device
@@ -171,10 +231,11 @@ extern "C" ulsnn_status_t ulsnn_sgemm_workspace_bytes(char transA, char transB, 
                                                       ulsnn_math_t math, size_t* bytes) {
     bool ta, tb;
     if (!bytes || !parse_trans(transA, &ta) || !parse_trans(transB, &tb) || M < 0 || N < 0 || K < 0) return ULSNN_ERR_INVALID_ARG;
-    if ((int)math < 0 || (int)math > 2) return ULSNN_ERR_INVALID_ARG;
+    if ((int)math < 0 || (int)math > 3) return ULSNN_ERR_INVALID_ARG;
     *bytes = 0;
     if (M == 0 || N == 0 || K == 0) return ULSNN_OK;
     SgemmArgs a{ta, tb, M, N, K, 1.f, 0.f, nullptr, ta ? M : K, nullptr, tb ? K : N, nullptr, N};
+    if (math == ULSNN_MATH_BF16) { *bytes = sgemm_need(a, math); return ULSNN_OK; }
     a.lda = round_up(a.lda, 4); a.ldb = round_up(a.ldb, 4);       // an addressable stand-in for the tile-width query
     GemmDesc d = sgemm_desc(a);
     size_t w = sgemm_ws_for(d, false);
@@ -190,7 +251,7 @@ extern "C" ulsnn_status_t ulsnn_sgemm_ex(char transA, char transB, int64_t M, in
     SgemmArgs a{false, false, M, N, K, alpha, beta, A, lda, B, ldb, C, ldc};
     ulsnn_status_t st = validate_sgemm(transA, transB, M, N, K, lda, ldb, ldc, &a.ta, &a.tb);
     if (st != ULSNN_OK) return st;
-    if ((int)math < 0 || (int)math > 2) return ULSNN_ERR_INVALID_ARG;
+    if ((int)math < 0 || (int)math > 3) return ULSNN_ERR_INVALID_ARG;
     if (M == 0 || N == 0) return ULSNN_OK;
     if ((st = check_arch()) != ULSNN_OK) return st;
     return sgemm_impl(a, math, workspace, workspace_bytes, (cudaStream_t)stream);
@@ -262,13 +323,12 @@ extern "C" ulsnn_status_t ulsnn_sgemm_noalloc(char transA, char transB, int64_t 
     SgemmArgs a{false, false, M, N, K, alpha, beta, A, lda, B, ldb, C, ldc};
     ulsnn_status_t st = validate_sgemm(transA, transB, M, N, K, lda, ldb, ldc, &a.ta, &a.tb);
     if (st != ULSNN_OK) return st;
-    if ((int)math < 0 || (int)math > 2) return ULSNN_ERR_INVALID_ARG;
+    if ((int)math < 0 || (int)math > 3) return ULSNN_ERR_INVALID_ARG;
     if (M == 0 || N == 0) return ULSNN_OK;
     size_t need = 0;
     if (K > 0 && alpha != 0.f && A && B && C) {
         // the same slice plan as ulsnn_sgemm_ex makes for these operands, so the two give the same bits
-        GemmDesc d = sgemm_desc(a);
-        need = sgemm_ws_for(d, use_tc(d, math));
+        need = sgemm_need(a, math);
     }
     if (need > (size_t)ULSNN_NOALLOC_SCRATCH_BYTES) return ULSNN_ERR_TOO_LARGE;
     if ((st = check_arch()) != ULSNN_OK) return st;

@@ -1,6 +1,7 @@
 // Shared declarations of the library's translation units (host + device).
 #pragma once
 #include <cuda_runtime.h>
+#include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
 #include "../../include/ulsnn.h"
@@ -57,6 +58,29 @@ struct GemmDesc {
     float* partials; int64_t ldp;        // partials[(s*M + i)*ldp + j]
 };
 
+// One product of the 16-bit engine: operands stored as bfloat16, fp32 accumulation.  The epilogues are those of
+// GemmDesc, except that activations, stored exponentials and deltas (BIAS_TANH, LOGITS, TANHP) are written as
+// bfloat16 to Ch, and that the transcendental functions are the hardware approximations.
+struct HalfGemmDesc {
+    int64_t M, N, K;
+    const __nv_bfloat16* A; int64_t a_sm, a_sk;   // A(i,k) = A[i*a_sm + k*a_sk]  (one of the strides is 1)
+    const __nv_bfloat16* B; int64_t b_sk, b_sn;   // B(k,j) = B[k*b_sk + j*b_sn]
+    int epi;                  // EPI_SGEMM, EPI_BIAS_TANH, EPI_LOGITS, EPI_TANHP or EPI_PARTIAL
+    float* C; int64_t ldc;    // SGEMM: fp32 output
+    float alpha, beta;
+    __nv_bfloat16* Ch; int64_t ldch;     // BIAS_TANH, LOGITS (may be null: statistics only), TANHP: bfloat16 output
+    const float* bias;        // [N]  BIAS_TANH, LOGITS
+    int ones_cols;            // BIAS_TANH: Ch[:, N] = 1 and Ch[:, N+1 .. N+ones_cols) = 0
+    const __nv_bfloat16* Hm; int64_t ldh;        // TANHP
+    const int32_t* labels;    // LOGITS
+    float2* stats; int64_t stats_ld;     // LOGITS: stats[row*stats_ld + 2*col_tile + h], h = 0, 1: (max, sum exp(z - max)) over
+                                         // the even (odd) 64-column blocks of the tile; (-inf, 0) when there is none
+    float* zlabel;
+    float* chunk_max; int64_t chunk_ld;  // LOGITS: as in GemmDesc
+    int splits; int64_t k_per_split;     // EPI_PARTIAL; k_per_split is a multiple of hg_k_granule()
+    float* partials; int64_t ldp;
+};
+
 // Device status word values (0 = fine).
 enum : int { DEV_OK = 0, DEV_TIMEOUT = 1 };
 
@@ -79,7 +103,23 @@ int tc_colsum_groups();
 int simt_colsum_groups();
 ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stream);
 // device status word shared by all kernels of the library on the current device
+int* device_status_word();      // its device address (null if it cannot be had)
 ulsnn_status_t device_status_fetch_and_clear(cudaStream_t stream, int* word);
+
+// 16-bit tcgen05 engine (bf16_gemm.cu): operands need 16-byte aligned bases and leading dimensions that are
+// multiples of 8 elements
+bool hg_gemm_supported(const HalfGemmDesc& d);
+int hg_tile_m(const HalfGemmDesc& d);
+int hg_tile_n(const HalfGemmDesc& d);
+int hg_slots(const HalfGemmDesc& d);
+int hg_k_granule();
+ulsnn_status_t hg_gemm_launch(const HalfGemmDesc& d, cudaStream_t stream);
+// dst[r][j] = bf16(src[r][j]), j < cols; dst[r][cols] = 1 when `ones`; the rest of each row up to ldd (a multiple of 8) = 0
+ulsnn_status_t launch_to_bf16(const float* src, int64_t rows, int64_t cols, int64_t lds, __nv_bfloat16* dst, int64_t ldd,
+                              int ones, cudaStream_t stream);
+// in place: stored exponentials -> bf16(e * scale[pattern][class/32] - [label == class]), zero beyond n_classes
+ulsnn_status_t launch_delta_bf16(__nv_bfloat16* E, int64_t lde, const float* scale, int64_t scale_ld, const int32_t* labels,
+                                 int64_t n, int64_t n_classes, cudaStream_t stream);
 
 // reductions and small kernels (reduce.cu)
 // out[i*ldo + j] = alpha * sum_s parts[(s*M + i)*ldp + j] + beta*out   for j < N;   if bias_out: column N goes to

@@ -4,7 +4,8 @@ import torch
 
 from paper_1911_05181_b200 import binding as ul
 
-TOL = {ul.MATH_3XTF32: 1e-5, ul.MATH_FP32_SIMT: 1e-5, ul.MATH_TF32: 5e-3}   # relative L2, per tensor
+# relative L2, per tensor; the 16-bit mode keeps 8 mantissa bits against TF32's 10: four times its tolerance
+TOL = {ul.MATH_3XTF32: 1e-5, ul.MATH_FP32_SIMT: 1e-5, ul.MATH_TF32: 5e-3, ul.MATH_BF16: 2e-2}
 
 
 def dev(a):

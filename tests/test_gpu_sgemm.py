@@ -10,7 +10,7 @@ from helpers import TOL, gpu_sgemm, dev
 
 pytestmark = pytest.mark.gpu
 
-MATHS = [ul.MATH_FP32_SIMT, ul.MATH_3XTF32, ul.MATH_TF32]
+MATHS = [ul.MATH_FP32_SIMT, ul.MATH_3XTF32, ul.MATH_TF32, ul.MATH_BF16]
 
 
 def _stored(trans_a, trans_b, M, N, K, pad, seed=1):
