@@ -3,7 +3,7 @@
 products with their fixed-order reduction, then the plain step W -= lr*grad) on synthetic data shaped like
 the paper's 400-480-3203 character-recognition network.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--math 3xtf32|tf32|simt] [--workload config3|config1|config5]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--math 3xtf32|tf32|simt|bf16] [--workload config3|config1|config5]
     python bench.py --impl reference ...      # times the CPU checker on the host cores instead
 
 One "step" = one error-and-gradient evaluation of one batch plus the parameter step.  Flops are counted with the
@@ -35,7 +35,7 @@ WORKLOADS = {
     "config4": ([400, 480, 3203], 9_000_000, 3),
 }
 CHUNK = {"config4": 131072}
-MATH = {"3xtf32": 0, "tf32": 1, "simt": 2}
+MATH = {"3xtf32": 0, "tf32": 1, "simt": 2, "bf16": 3}
 NOMINAL_TF32_OVER_BF16 = 0.5        # dense TF32 tensor rate is half the BF16 rate
 # DRAM bytes per launch of the dominant kernel from one ncu capture (profiles/tc_gemm_3xtf32_config3.md: measured at
 # 16384 patterns and scaled by the pattern count).  Only reported while the library still is the version the
@@ -187,7 +187,8 @@ def run_sgemm_sweep(args):
         return 0
     math_mode = MATH[args.math]
     peaks = load_peaks()
-    tf32_peak = peaks["bf16_tflops_sustained"] * NOMINAL_TF32_OVER_BF16
+    # tensor peak of the mode's operand type: the measured bf16 rate, halved for TF32 (nominal ratio)
+    tf32_peak = peaks["bf16_tflops_sustained"] * (1.0 if args.math == "bf16" else NOMINAL_TF32_OVER_BF16)
     mult = 3.0 if args.math == "3xtf32" else 1.0
     stream = torch.cuda.current_stream()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")          # > L2: written between timed calls
@@ -221,7 +222,7 @@ def run_sgemm_sweep(args):
     big = [r for r in rows if r["M"] == 8192][0]
     line = {"metric": "sgemm_gflops", "value": big["logical_tflops"] * 1e3, "unit": "GFLOP/s", "n_gpus": 1, "steps": 8,
             "warmup": 3, "ms_per_step": big["ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
+            "dtype": "bf16" if args.math == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": "sgemm sweep (alpha 1, beta 0, uniform [-1,1), seed 1); value = NN 8192^3", "math": args.math,
                        "l2": "a 256 MB buffer is overwritten between timed calls"},
             "sweep": rows, "peak_tflops": tf32_peak, "gpu_launches": int(sum(ul.launch_counts().values()))}
@@ -421,15 +422,18 @@ def main():
         on_tensor = args.math != "simt" and counts["tc_gemm"] > 0
         if on_tensor:
             mult = 3.0 if args.math == "3xtf32" else 1.0
-            peak = peaks["bf16_tflops_sustained"] * NOMINAL_TF32_OVER_BF16
+            half = args.math == "bf16"
+            peak = peaks["bf16_tflops_sustained"] * (1.0 if half else NOMINAL_TF32_OVER_BF16)
+            esize = 2.0 if half else 4.0
             achieved = mult * logical / (ms_k * 1e-3) / 1e12
             roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                         "traffic": (NCU_TRAFFIC.get((args.workload, args.math, (M, N, K)))
                                     if ul.version() == NCU_TRAFFIC["library_version"] and args.patterns <= 0 else None),
-                        "algorithmic_bytes": 4.0 * (M * K + K * N) + (4.0 * M * N if K <= 8192 else 0.0),
-                        "kernel": "tc_gemm M=%d N=%d K=%d" % (M, N, K), "ms": ms_k,
+                        "algorithmic_bytes": esize * (M * K + K * N) + (esize * M * N if K <= 8192 else 0.0),
+                        "kernel": "%s M=%d N=%d K=%d" % ("bf16_gemm" if half else "tc_gemm", M, N, K), "ms": ms_k,
                         "flops_counted": "%gx 2MNK" % mult, "logical_tflops": logical / (ms_k * 1e-3) / 1e12,
-                        "peak_source": "%s cuBLAS bf16 sustained x 0.5 (nominal TF32:BF16)" % peaks["_source"]}
+                        "peak_source": ("%s cuBLAS bf16 sustained" if half else
+                                        "%s cuBLAS bf16 sustained x 0.5 (nominal TF32:BF16)") % peaks["_source"]}
         else:
             sm_mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
             peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12      # FFMA lanes x 2 flops x clock seen during the run
@@ -447,7 +451,7 @@ def main():
     line = {
         "metric": "gradient_eval_gflops", "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "bf16" if args.math == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": "%s: %s MLP, %d patterns per GPU, seed %d" % (args.workload, "-".join(map(str, sizes)), batch, seed),
                    "math": args.math, "head": args.head, "global_batch": batch * world, "parallelism": "dp%d" % world,
                    "l2": "no flush: inputs and intermediates of a step (X %.0f MB, logits %.0f MB) exceed the 126 MB L2"
@@ -467,11 +471,13 @@ def main():
         "device_status": status,
         "peaks": {k: peaks.get(k) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "_source")},
     }
-    tf32_peak = peaks["bf16_tflops_sustained"] * NOMINAL_TF32_OVER_BF16 * 1e3   # GFLOP/s
+    # tensor peak of the mode's operand type: the measured bf16 rate, halved (nominal ratio) for the TF32 modes
+    half = args.math == "bf16"
+    tf32_peak = peaks["bf16_tflops_sustained"] * (1.0 if half else NOMINAL_TF32_OVER_BF16) * 1e3   # GFLOP/s
     mult = 3.0 if args.math == "3xtf32" else 1.0
     line["pct_of_tf32_peak"] = {"logical": 100.0 * value / world / tf32_peak,
                                 "tensor_pipe": 100.0 * mult * value / world / tf32_peak if args.math != "simt" else None,
-                                "peak_gflops": tf32_peak}
+                                "peak_gflops": tf32_peak, "peak_dtype": "bf16" if half else "tf32"}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -369,6 +369,14 @@ struct ulsnn_mlp {
     float* partials;
     size_t partials_bytes;
     size_t total_bytes;
+    // 16-bit mode: bfloat16 copies of the batch and the weights (rebuilt every call), activations, deltas and stored
+    // exponentials.  Activation rows (the batch included) end in a ones column, so that every bias gradient is a
+    // column of a weight-gradient product.
+    __nv_bfloat16* Xb; int64_t ldxb;
+    __nv_bfloat16* Wb[MAX_LAYERS]; int64_t ldwb[MAX_LAYERS];
+    __nv_bfloat16* Hb[MAX_LAYERS + 1]; int64_t ldhb[MAX_LAYERS + 1];
+    __nv_bfloat16* Db[MAX_LAYERS + 1]; int64_t lddb[MAX_LAYERS + 1];
+    __nv_bfloat16* Eb; int64_t ldeb;
     // optional per-product timing
     bool timing;
     int n_phases;                       // products launched so far by the call in flight
@@ -400,7 +408,59 @@ size_t wgrad_partial_bound(const int32_t* sizes, int w, int64_t B) {
     return (size_t)smax * (size_t)d.M * (size_t)ldp * sizeof(float);
 }
 
+// 16-bit mode: split-K scratch bound for dW_w, M = sizes[w+1], N = sizes[w] + 1 (ones column), any n <= B
+size_t wgrad_partial_bound_bf16(const int32_t* sizes, int w, int64_t B) {
+    HalfGemmDesc d{};
+    d.M = sizes[w + 1]; d.N = sizes[w] + 1; d.K = B;
+    d.a_sm = 1; d.a_sk = 8; d.b_sk = 8; d.b_sn = 1;
+    const int64_t ldp = round_up(d.N, 4);
+    int64_t smax = (B + SLICE_CAP - 1) / SLICE_CAP;
+    const int64_t tiles = ((d.M + hg_tile_m(d) - 1) / hg_tile_m(d)) * ((d.N + hg_tile_n(d) - 1) / hg_tile_n(d));
+    const int64_t slots = hg_slots(d);
+    if (tiles < slots && B >= 1024) {
+        int64_t f = (2 * slots + tiles - 1) / tiles;
+        if (f > B / 512) f = B / 512;
+        if (f > smax) smax = f;
+    }
+    if (smax < 1) smax = 1;
+    return (size_t)smax * (size_t)d.M * (size_t)ldp * sizeof(float);
+}
+
+ulsnn_status_t layout_bf16(ulsnn_mlp* h, char* base) {
+    const int L = h->L; const int64_t B = h->max_patterns;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* p = base ? base + off : nullptr; off += align256(bytes); return p; };
+    h->ldxb = round_up((int64_t)h->sizes[0] + 1, 8);
+    h->Xb = (__nv_bfloat16*)take((size_t)B * h->ldxb * 2);
+    for (int l = 1; l < L; ++l) {
+        h->ldhb[l] = round_up((int64_t)h->sizes[l] + 1, 8);
+        h->lddb[l] = round_up((int64_t)h->sizes[l], 8);
+        h->Hb[l] = (__nv_bfloat16*)take((size_t)B * h->ldhb[l] * 2);
+        h->Db[l] = (__nv_bfloat16*)take((size_t)B * h->lddb[l] * 2);
+    }
+    for (int l = 0; l < L; ++l) {
+        h->ldwb[l] = round_up((int64_t)h->sizes[l], 8);
+        h->Wb[l] = (__nv_bfloat16*)take((size_t)h->sizes[l + 1] * h->ldwb[l] * 2);
+    }
+    h->ldeb = round_up((int64_t)h->sizes[L], 8);
+    h->Eb = (__nv_bfloat16*)take((size_t)B * h->ldeb * 2);
+    h->stats_ld = 2 * (((int64_t)h->sizes[L] + 63) / 64);       // two entries per column tile, tiles at least 64 wide
+    h->stats = (float2*)take((size_t)B * h->stats_ld * sizeof(float2));
+    h->lse = (float*)take((size_t)B * sizeof(float));
+    h->chunk_ld = round_up(((int64_t)h->sizes[L] + 31) / 32, 8);
+    h->chunk_tab = (float*)take((size_t)B * h->chunk_ld * sizeof(float));
+    h->zlabel = (float*)take((size_t)B * sizeof(float));
+    h->loss_parts = (double*)take((size_t)(rowstats_blocks(B) + 1) * sizeof(double));
+    size_t pb = 0;
+    for (int w = 0; w < L; ++w) { const size_t b = wgrad_partial_bound_bf16(h->sizes, w, B); if (b > pb) pb = b; }
+    h->partials_bytes = align256(pb);
+    h->partials = (float*)take(pb);
+    h->total_bytes = off;
+    return ULSNN_OK;
+}
+
 ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
+    if (h->math == ULSNN_MATH_BF16) return layout_bf16(h, base);
     const int L = h->L; const int64_t B = h->max_patterns;
     size_t off = 0;
     auto take = [&](size_t bytes) { char* p = base ? base + off : nullptr; off += align256(bytes); return p; };
@@ -444,7 +504,7 @@ ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
 
 ulsnn_status_t check_desc(const ulsnn_mlp_desc_t* d) {
     if (!d || !d->sizes || d->n_layers < 1 || d->n_layers > MAX_LAYERS || d->max_patterns < 1) return ULSNN_ERR_INVALID_ARG;
-    if ((int)d->math < 0 || (int)d->math > 2) return ULSNN_ERR_INVALID_ARG;
+    if ((int)d->math < 0 || (int)d->math > 3) return ULSNN_ERR_INVALID_ARG;
     for (int l = 0; l <= d->n_layers; ++l) if (d->sizes[l] < 1 || d->sizes[l] > (1 << 20)) return ULSNN_ERR_INVALID_ARG;
     if (d->max_patterns > ((int64_t)1 << 31) - 256) return ULSNN_ERR_TOO_LARGE;
     return ULSNN_OK;
@@ -467,17 +527,24 @@ void set_weight_operand(ulsnn_mlp* h, GemmDesc& d, const float* const* W, int w)
     }
 }
 
-// run_gemm bracketed by events when the handle's timing is on
-ulsnn_status_t timed_gemm(ulsnn_mlp* h, const GemmDesc& d, cudaStream_t stream) {
-    if (!h->timing || h->n_phases >= 3 * MAX_LAYERS) return run_gemm(d, h->math, stream);
+// a product's launch bracketed by events when the handle's timing is on
+template <class Launch>
+ulsnn_status_t timed_product(ulsnn_mlp* h, int64_t M, int64_t N, int64_t K, cudaStream_t stream, Launch launch) {
+    if (!h->timing || h->n_phases >= 3 * MAX_LAYERS) return launch();
     const int i = h->n_phases++;
-    h->phase_mnk[3 * i] = d.M; h->phase_mnk[3 * i + 1] = d.N; h->phase_mnk[3 * i + 2] = d.K;
+    h->phase_mnk[3 * i] = M; h->phase_mnk[3 * i + 1] = N; h->phase_mnk[3 * i + 2] = K;
     const size_t slot = (size_t)((h->timed_calls - 1) % TIMING_SLOTS);
     cudaEvent_t* e = &h->ev[(slot * 3 * MAX_LAYERS + i) * 2];
     if (cudaEventRecord(e[0], stream) != cudaSuccess) return ULSNN_ERR_CUDA;
-    ulsnn_status_t st = run_gemm(d, h->math, stream);
+    ulsnn_status_t st = launch();
     if (cudaEventRecord(e[1], stream) != cudaSuccess) return ULSNN_ERR_CUDA;
     return st;
+}
+ulsnn_status_t timed_gemm(ulsnn_mlp* h, const GemmDesc& d, cudaStream_t stream) {
+    return timed_product(h, d.M, d.N, d.K, stream, [&] { return run_gemm(d, h->math, stream); });
+}
+ulsnn_status_t timed_gemm(ulsnn_mlp* h, const HalfGemmDesc& d, cudaStream_t stream) {
+    return timed_product(h, d.M, d.N, d.K, stream, [&] { return hg_gemm_launch(d, stream); });
 }
 
 // The forward products: hidden layers with bias + tanh fused, then the logits with their row statistics.
@@ -538,6 +605,86 @@ ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* 
     if (tg.T) return launch_rowsums(h->stats, h->stats_ld, tiles, n, h->loss_parts, accumulate, loss_out, stream);
     return launch_rowstats(h->stats, h->stats_ld, tiles, h->zlabel, n, h->lse, d.chunk_max, h->chunk_ld,
                            (int)(((int64_t)h->sizes[L] + 31) / 32), h->loss_parts, accumulate, loss_out, stream);
+}
+
+// ---- 16-bit mode (softmax head).  The batch and the weights are rounded to bfloat16 first; every product then reads
+// and writes bfloat16 (fp32 accumulators, fp32 statistics, loss and gradients).
+ulsnn_status_t forward_bf16(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
+                            const int32_t* labels, int64_t n, bool keep, int accumulate, double* loss_out, cudaStream_t stream) {
+    const int L = h->L;
+    h->n_phases = 0;
+    if (h->timing) h->timed_calls++;
+    ulsnn_status_t st = launch_to_bf16(X, n, h->sizes[0], ldx, h->Xb, h->ldxb, 1, stream);
+    if (st != ULSNN_OK) return st;
+    for (int l = 0; l < L; ++l)
+        if ((st = launch_to_bf16(W[l], h->sizes[l + 1], h->sizes[l], h->sizes[l], h->Wb[l], h->ldwb[l], 0, stream)) != ULSNN_OK) return st;
+    const __nv_bfloat16* in = h->Xb; int64_t ld_in = h->ldxb;
+    for (int l = 1; l < L; ++l) {
+        HalfGemmDesc d{};
+        d.M = n; d.N = h->sizes[l]; d.K = h->sizes[l - 1];
+        d.A = in; d.a_sm = ld_in; d.a_sk = 1;
+        d.B = h->Wb[l - 1]; d.b_sk = 1; d.b_sn = h->ldwb[l - 1];
+        d.Ch = h->Hb[l]; d.ldch = h->ldhb[l];
+        d.epi = EPI_BIAS_TANH; d.bias = b[l - 1]; d.ones_cols = (int)(h->ldhb[l] - d.N);
+        d.splits = 1; d.k_per_split = d.K;
+        if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
+        in = h->Hb[l]; ld_in = h->ldhb[l];
+    }
+    HalfGemmDesc d{};
+    d.M = n; d.N = h->sizes[L]; d.K = h->sizes[L - 1];
+    d.A = in; d.a_sm = ld_in; d.a_sk = 1;
+    d.B = h->Wb[L - 1]; d.b_sk = 1; d.b_sn = h->ldwb[L - 1];
+    d.Ch = keep ? h->Eb : nullptr; d.ldch = h->ldeb;
+    d.epi = EPI_LOGITS; d.bias = b[L - 1]; d.labels = labels;
+    d.stats = h->stats; d.stats_ld = h->stats_ld; d.zlabel = h->zlabel;
+    d.chunk_max = keep ? h->chunk_tab : nullptr; d.chunk_ld = h->chunk_ld;
+    d.splits = 1; d.k_per_split = d.K;
+    const int entries = 2 * (int)((d.N + hg_tile_n(d) - 1) / hg_tile_n(d));
+    if (entries > h->stats_ld) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
+    if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
+    return launch_rowstats(h->stats, h->stats_ld, entries, h->zlabel, n, h->lse, d.chunk_max, h->chunk_ld,
+                           (int)(((int64_t)h->sizes[L] + 31) / 32), h->loss_parts, accumulate, loss_out, stream);
+}
+
+ulsnn_status_t gradient_bf16(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
+                             const int32_t* labels, int64_t n, int accumulate, float* const* dW, float* const* db,
+                             double* loss_out, cudaStream_t stream) {
+    const int L = h->L;
+    ulsnn_status_t st = forward_bf16(h, W, b, X, ldx, labels, n, true, accumulate, loss_out, stream);
+    if (st != ULSNN_OK) return st;
+    // delta_L = softmax - onehot, in place over the stored exponentials
+    if ((st = launch_delta_bf16(h->Eb, h->ldeb, h->chunk_tab, h->chunk_ld, labels, n, h->sizes[L], stream)) != ULSNN_OK) return st;
+    // delta_l = (1 - H_l*H_l) * (delta_{l+1} W_{l+1})   (H_D of Section 4.2)
+    for (int l = L - 1; l >= 1; --l) {
+        HalfGemmDesc d{};
+        d.M = n; d.N = h->sizes[l]; d.K = h->sizes[l + 1];
+        if (l + 1 == L) { d.A = h->Eb; d.a_sm = h->ldeb; } else { d.A = h->Db[l + 1]; d.a_sm = h->lddb[l + 1]; }
+        d.a_sk = 1;
+        d.B = h->Wb[l]; d.b_sk = h->ldwb[l]; d.b_sn = 1;
+        d.Ch = h->Db[l]; d.ldch = h->lddb[l];
+        d.epi = EPI_TANHP; d.Hm = h->Hb[l]; d.ldh = h->ldhb[l];
+        d.splits = 1; d.k_per_split = d.K;
+        if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
+    }
+    // dW_w = delta_{w+1}^T [act_w | 1]: the last column is db_w
+    const float beta = accumulate ? 1.f : 0.f;
+    for (int w = L - 1; w >= 0; --w) {
+        HalfGemmDesc d{};
+        d.M = h->sizes[w + 1]; d.N = h->sizes[w] + 1; d.K = n;
+        if (w + 1 == L) { d.A = h->Eb; d.a_sk = h->ldeb; } else { d.A = h->Db[w + 1]; d.a_sk = h->lddb[w + 1]; }
+        d.a_sm = 1;
+        if (w >= 1) { d.B = h->Hb[w]; d.b_sk = h->ldhb[w]; } else { d.B = h->Xb; d.b_sk = h->ldxb; }
+        d.b_sn = 1;
+        d.epi = EPI_PARTIAL;
+        const int64_t tiles = ((d.M + hg_tile_m(d) - 1) / hg_tile_m(d)) * ((d.N + hg_tile_n(d) - 1) / hg_tile_n(d));
+        const SplitPlan p = plan_splits(tiles, d.K, hg_slots(d), hg_k_granule());
+        d.splits = p.splits; d.k_per_split = p.k_per_split;
+        d.ldp = round_up(d.N, 4); d.partials = h->partials;
+        if ((size_t)p.splits * (size_t)d.M * (size_t)d.ldp * sizeof(float) > h->partials_bytes) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
+        if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
+        if ((st = launch_splitk_reduce(d.partials, p.splits, d.M, h->sizes[w], d.ldp, 1.f, beta, dW[w], h->sizes[w], db[w], stream)) != ULSNN_OK) return st;
+    }
+    return ULSNN_OK;
 }
 
 ulsnn_status_t check_call(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
@@ -627,7 +774,9 @@ ulsnn_status_t forward_call(ulsnn_mlp_t* h, const float* const* W, const float* 
     if (st != ULSNN_OK) return st;
     if (tg.T && n > 0 && tg.ldt < h->sizes[h->L]) return ULSNN_ERR_INVALID_ARG;
     if ((st = check_arch()) != ULSNN_OK) return st;
+    if (h->math == ULSNN_MATH_BF16 && tg.T) return ULSNN_ERR_INVALID_ARG;     // the 16-bit mode has the softmax head only
     if (n == 0) return launch_zero_f64(loss_out, 1, stream);
+    if (h->math == ULSNN_MATH_BF16) return forward_bf16(h, W, b, X, ldx, tg.labels, n, false, 0, loss_out, stream);
     return forward(h, W, b, X, ldx, tg, n, false, 0, loss_out, stream);
 }
 
@@ -642,6 +791,7 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
     const bool sse = tg.T != nullptr;
     const int32_t* labels = tg.labels;
     for (int l = 0; l < L; ++l) if (!dW[l] || !db[l]) return ULSNN_ERR_INVALID_ARG;
+    if (h->math == ULSNN_MATH_BF16 && sse) return ULSNN_ERR_INVALID_ARG;
     if ((st = check_arch()) != ULSNN_OK) return st;
     if (n == 0) {
         if (accumulate) return ULSNN_OK;
@@ -651,6 +801,7 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
         }
         return launch_zero_f64(loss_out, 1, stream);
     }
+    if (h->math == ULSNN_MATH_BF16) return gradient_bf16(h, W, b, X, ldx, labels, n, accumulate, dW, db, loss_out, stream);
     if ((st = forward(h, W, b, X, ldx, tg, n, true, accumulate, loss_out, stream)) != ULSNN_OK) return st;
 
     int64_t colsum_rows = 0;

@@ -12,7 +12,7 @@ from helpers import TOL, GpuNet, dev
 
 pytestmark = pytest.mark.gpu
 
-MATHS = [ul.MATH_FP32_SIMT, ul.MATH_3XTF32, ul.MATH_TF32]
+MATHS = [ul.MATH_FP32_SIMT, ul.MATH_3XTF32, ul.MATH_TF32, ul.MATH_BF16]
 
 
 def _net(seed, sizes, bias_scale=0.2):

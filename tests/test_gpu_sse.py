@@ -89,3 +89,11 @@ def test_bad_arguments():
     assert g.net.gradient_sse(g.W, g.b, X, 8, T, 2, 4, False, g.dW, g.db, g.loss, check=False) == ul.ERR_INVALID_ARG   # ldt < n_L
     assert g.net.gradient_sse(g.W, g.b, X, 8, None, 3, 4, False, g.dW, g.db, g.loss, check=False) == ul.ERR_INVALID_ARG
     assert g.net.forward_sse(g.W, g.b, X, 8, T, 3, 17, g.loss, check=False) == ul.ERR_INVALID_ARG                     # n > max
+
+
+def test_sixteen_bit_mode_has_no_squared_error_head():
+    sizes = [8, 4, 3]
+    g = GpuNet(sizes, ul.MATH_BF16, 16); g.set_params(*_net(43, sizes))
+    X = dev(np.zeros((4, 8), np.float32)); T = dev(np.zeros((4, 3), np.float32))
+    assert g.net.gradient_sse(g.W, g.b, X, 8, T, 3, 4, False, g.dW, g.db, g.loss, check=False) == ul.ERR_INVALID_ARG
+    assert g.net.forward_sse(g.W, g.b, X, 8, T, 3, 4, g.loss, check=False) == ul.ERR_INVALID_ARG
