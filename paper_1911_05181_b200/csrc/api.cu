@@ -16,6 +16,7 @@ namespace {
 constexpr int MAX_LAYERS = 16;
 constexpr int TIMING_SLOTS = 64;        // per-product timings are kept for this many most recent calls
 constexpr int64_t SLICE_CAP = 4096;     // longest run of patterns summed in one fp32 accumulator
+constexpr int64_t SLICE_CAP_BF16 = 8192;    // 16-bit mode: the operands' rounding dwarfs the accumulator's, fewer partials to reduce
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -55,8 +56,8 @@ struct SplitPlan { int splits; int64_t k_per_split; };
 
 // Fixed by the shapes only.  Slices are at most SLICE_CAP long once K is large (bounds the fp32 rounding of a
 // long sum), and short-and-wide products get enough slices to fill the GPU.
-SplitPlan plan_splits(int64_t tiles, int64_t K, int64_t slots, int64_t granule = 32) {
-    int64_t s_acc = (K > 2 * SLICE_CAP) ? (K + SLICE_CAP - 1) / SLICE_CAP : 1;
+SplitPlan plan_splits(int64_t tiles, int64_t K, int64_t slots, int64_t granule = 32, int64_t cap = SLICE_CAP) {
+    int64_t s_acc = (K > 2 * cap) ? (K + cap - 1) / cap : 1;
     int64_t s_fill = 1;
     if (tiles < slots && K >= 1024) {
         s_fill = (2 * slots + tiles - 1) / tiles;
@@ -163,7 +164,7 @@ HalfSgemmPlan half_sgemm_plan(const SgemmArgs& a) {
     pl.b_bytes = align256((size_t)pl.b_rows * pl.ldb * 2);
     const HalfGemmDesc d = half_sgemm_desc(a, pl, nullptr, nullptr);
     const int64_t tiles = ((d.M + hg_tile_m(d) - 1) / hg_tile_m(d)) * ((d.N + hg_tile_n(d) - 1) / hg_tile_n(d));
-    pl.sp = plan_splits(tiles, d.K, hg_slots(d), hg_k_granule());
+    pl.sp = plan_splits(tiles, d.K, hg_slots(d), hg_k_granule(), SLICE_CAP_BF16);
     pl.ldp = round_up(d.N, 4);
     pl.part_bytes = pl.sp.splits <= 1 ? 0 : align256((size_t)pl.sp.splits * (size_t)d.M * (size_t)pl.ldp * sizeof(float));
     return pl;
@@ -414,7 +415,7 @@ size_t wgrad_partial_bound_bf16(const int32_t* sizes, int w, int64_t B) {
     d.M = sizes[w + 1]; d.N = sizes[w] + 1; d.K = B;
     d.a_sm = 1; d.a_sk = 8; d.b_sk = 8; d.b_sn = 1;
     const int64_t ldp = round_up(d.N, 4);
-    int64_t smax = (B + SLICE_CAP - 1) / SLICE_CAP;
+    int64_t smax = (B + SLICE_CAP_BF16 - 1) / SLICE_CAP_BF16;
     const int64_t tiles = ((d.M + hg_tile_m(d) - 1) / hg_tile_m(d)) * ((d.N + hg_tile_n(d) - 1) / hg_tile_n(d));
     const int64_t slots = hg_slots(d);
     if (tiles < slots && B >= 1024) {
@@ -677,7 +678,7 @@ ulsnn_status_t gradient_bf16(ulsnn_mlp* h, const float* const* W, const float* c
         d.b_sn = 1;
         d.epi = EPI_PARTIAL;
         const int64_t tiles = ((d.M + hg_tile_m(d) - 1) / hg_tile_m(d)) * ((d.N + hg_tile_n(d) - 1) / hg_tile_n(d));
-        const SplitPlan p = plan_splits(tiles, d.K, hg_slots(d), hg_k_granule());
+        const SplitPlan p = plan_splits(tiles, d.K, hg_slots(d), hg_k_granule(), SLICE_CAP_BF16);
         d.splits = p.splits; d.k_per_split = p.k_per_split;
         d.ldp = round_up(d.N, 4); d.partials = h->partials;
         if ((size_t)p.splits * (size_t)d.M * (size_t)d.ldp * sizeof(float) > h->partials_bytes) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
@@ -903,11 +904,13 @@ extern "C" ulsnn_status_t ulsnn_sgd_step(ulsnn_mlp_t* h, float* const* W, float*
     for (int l = 0; l < h->L; ++l) if (!W[l] || !b[l] || !dW[l] || !db[l]) return ULSNN_ERR_INVALID_ARG;
     ulsnn_status_t st = check_arch();
     if (st != ULSNN_OK) return st;
+    SgdBatch batch{};
     for (int l = 0; l < h->L; ++l) {
-        if ((st = launch_sgd(W[l], dW[l], (int64_t)h->sizes[l] * h->sizes[l + 1], lr, (cudaStream_t)stream)) != ULSNN_OK) return st;
-        if ((st = launch_sgd(b[l], db[l], h->sizes[l + 1], lr, (cudaStream_t)stream)) != ULSNN_OK) return st;
+        batch.w[2 * l] = W[l]; batch.g[2 * l] = dW[l]; batch.n[2 * l] = (int64_t)h->sizes[l] * h->sizes[l + 1];
+        batch.w[2 * l + 1] = b[l]; batch.g[2 * l + 1] = db[l]; batch.n[2 * l + 1] = h->sizes[l + 1];
     }
-    return ULSNN_OK;
+    batch.count = 2 * h->L;
+    return launch_sgd_multi(batch, lr, (cudaStream_t)stream);
 }
 
 extern "C" ulsnn_status_t ulsnn_vec_dot_workspace_bytes(int64_t n, size_t* bytes) {

@@ -306,15 +306,15 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int n0 = nt * p.bn;
             const int cols_in = min(p.bn, (int)d.N - n0);
             const int nblk = (cols_in + 63) >> 6;           // 64-column blocks of this tile inside the matrix
-            if (!wait_bar(&ctrl->reg_full[acc], (tile_i >> 1) & 1, ctrl, p.status)) { ok = false; break; }
-            tc_fence_after();
             const int r0w = (mt * CG + rank) * BM + q * 32;
             const int64_t r = (int64_t)r0w + lane;
             const bool rv = r < d.M;
             float run_m = -INFINITY, run_s = 0.f, zl = 0.f;
             bool have_zl = false;
             int lab = -1;
-            if (EPI == EPI_LOGITS && rv) lab = __ldg(d.labels + r);
+            if (EPI == EPI_LOGITS && rv) lab = __ldg(d.labels + r);        // asked for before the wait for the products
+            if (!wait_bar(&ctrl->reg_full[acc], (tile_i >> 1) & 1, ctrl, p.status)) { ok = false; break; }
+            tc_fence_after();
 
             // next staging block of this warp, free to be written
             auto next_block = [&]() -> uint8_t* {
@@ -328,6 +328,30 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             for (int blk64 = half; blk64 < nblk; blk64 += 2) {
                 uint32_t packed[32];                    // OUT16: this thread's 64 values of the block, as bf16 pairs
                 float cmax[2] = {0.f, 0.f};
+                // both 32-column chunks of the block and their biases are asked for before the first is used
+                uint32_t raw[2][32];
+                float bv[2][32];
+                const int nv64 = min(64, (int)d.N - (n0 + blk64 * 64));
+                tmem_ld32(tmem_base + acc * BN_MAX + (2 * blk64) * 32 + lane_off, raw[0]);
+                if (nv64 > 32) tmem_ld32(tmem_base + acc * BN_MAX + (2 * blk64 + 1) * 32 + lane_off, raw[1]);
+                if (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) {
+#pragma unroll
+                    for (int cc = 0; cc < 2; ++cc) {
+                        const int c0 = n0 + (2 * blk64 + cc) * 32;
+                        const int nvalid = max(0, min(32, (int)d.N - c0));
+                        if (bias_vec && nvalid == 32) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                const float4 bb = __ldg(reinterpret_cast<const float4*>(d.bias + c0 + j));
+                                bv[cc][j] = bb.x; bv[cc][j + 1] = bb.y; bv[cc][j + 2] = bb.z; bv[cc][j + 3] = bb.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) bv[cc][j] = (j < nvalid) ? __ldg(d.bias + c0 + j) : 0.f;
+                        }
+                    }
+                }
+                tmem_ld_wait();
 #pragma unroll
                 for (int cc = 0; cc < 2; ++cc) {
                     const int c = 2 * blk64 + cc;
@@ -335,16 +359,8 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const int nvalid = max(0, min(32, (int)d.N - c0));
                     const bool full = nvalid == 32;
                     float v[32];
-                    if (nvalid > 0) {
-                        uint32_t raw[32];
-                        tmem_ld32(tmem_base + acc * BN_MAX + c * 32 + lane_off, raw);
-                        tmem_ld_wait();
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = 0.f;
-                    }
+                    for (int j = 0; j < 32; ++j) v[j] = (nvalid > 0) ? __uint_as_float(raw[cc][j]) : 0.f;
 
                     if (EPI == EPI_SGEMM) {
                         if (d.beta != 0.f) {
@@ -367,25 +383,17 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                             for (int j = 0; j < 32; ++j) v[j] = d.alpha * v[j];
                         }
                     } else if (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) {
-                        if (nvalid > 0) {
-                            if (bias_vec && full) {
 #pragma unroll
-                                for (int j = 0; j < 32; j += 4) {
-                                    const float4 bb = __ldg(reinterpret_cast<const float4*>(d.bias + c0 + j));
-                                    v[j] += bb.x; v[j + 1] += bb.y; v[j + 2] += bb.z; v[j + 3] += bb.w;
-                                }
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) if (j < nvalid) v[j] += __ldg(d.bias + c0 + j);
-                            }
-                        }
+                        for (int j = 0; j < 32; ++j) v[j] += bv[cc][j];
                         if (EPI == EPI_BIAS_TANH) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = (j < nvalid) ? tanh_approx(v[j]) : 0.f;
                         } else if (nvalid > 0) {
-                            float cm = -INFINITY;
+                            // four interleaved chains each for the maximum and the sum (fixed order)
+                            float cm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) { if (j >= nvalid) v[j] = -INFINITY; cm = fmaxf(cm, v[j]); }
+                            for (int j = 0; j < 32; ++j) { if (j >= nvalid) v[j] = -INFINITY; cm4[j & 3] = fmaxf(cm4[j & 3], v[j]); }
+                            const float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
                             const float nm = fmaxf(run_m, cm);
                             if ((unsigned)(lab - c0) < (unsigned)nvalid) {
 #pragma unroll
@@ -394,9 +402,10 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                             }
                             // stored: exp(z - nm), nm noted per 32-class chunk; the same values make up the row sum
                             const float nm2 = nm * LOG2E;
-                            float s = 0.f;
+                            float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) { v[j] = (j < nvalid) ? ex2_approx(fmaf(v[j], LOG2E, -nm2)) : 0.f; s += v[j]; }
+                            for (int j = 0; j < 32; ++j) { v[j] = (j < nvalid) ? ex2_approx(fmaf(v[j], LOG2E, -nm2)) : 0.f; s4[j & 3] += v[j]; }
+                            const float s = (s4[0] + s4[1]) + (s4[2] + s4[3]);
                             run_s = (run_m == -INFINITY ? 0.f : run_s * ex2_approx((run_m - nm) * LOG2E)) + s;
                             run_m = nm;
                             cmax[cc] = nm;
@@ -476,7 +485,6 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                             }
                         } else if (rv) {
                             __nv_bfloat16* dst = d.Ch + r * d.ldch + c0;
-                            const int nv64 = min(64, (int)d.N - c0);
                             if (ch_vec && nv64 == 64) {
 #pragma unroll
                                 for (int j = 0; j < 8; ++j)

@@ -155,7 +155,9 @@ ulsnn_status_t launch_split_hilo(const float* x, int64_t n, float* hi, float* lo
 ulsnn_status_t launch_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out, cudaStream_t stream);
 ulsnn_status_t launch_dot(int64_t n, const float* x, const float* y, double* out, double* parts, cudaStream_t stream);
 int64_t dot_parts(int64_t n);
-ulsnn_status_t launch_sgd(float* w, const float* g, int64_t n, float lr, cudaStream_t stream);
+// w[t][i] -= lr * g[t][i] for `count` tensors in one launch
+struct SgdBatch { static constexpr int MAX = 32; float* w[MAX]; const float* g[MAX]; int64_t n[MAX]; int count; };
+ulsnn_status_t launch_sgd_multi(const SgdBatch& b, float lr, cudaStream_t stream);
 ulsnn_status_t launch_zero(float* p, int64_t n, cudaStream_t stream);
 ulsnn_status_t launch_zero_f64(double* p, int64_t n, cudaStream_t stream);
 ulsnn_status_t launch_scale_rows(float* C, int64_t M, int64_t N, int64_t ldc, float beta, cudaStream_t stream);

@@ -53,7 +53,7 @@ constexpr int RS_THREADS = 256;
 // One warp per pattern (each of a block's 8 warps takes 8 patterns in turn): the lanes combine the per-tile
 // (max, sum-exp) pairs -- every lane its tiles in index order, then a fixed shuffle tree -- into the log-sum-exp,
 // and turn the pattern's chunk maxima into the factors exp(m - lse).  lse - z_label is then summed over the
-// block's 64 patterns in a fixed tree.
+// block's 64 patterns in a fixed tree.  Everything a pattern needs from memory is asked for before the first use.
 constexpr int RS_ROWS = 64;
 __global__ void __launch_bounds__(RS_THREADS)
 rowstats_kernel(const float2* __restrict__ stats, int64_t stats_ld, int tiles,
@@ -62,30 +62,39 @@ rowstats_kernel(const float2* __restrict__ stats, int64_t stats_ld, int tiles,
                 double* __restrict__ block_partials) {
     __shared__ double red[RS_ROWS];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll 2
     for (int i = 0; i < RS_ROWS / 8; ++i) {
         const int row = warp * (RS_ROWS / 8) + i;
         const int64_t p = (int64_t)blockIdx.x * RS_ROWS + row;
         double term = 0.0;
         if (p < n) {                                        // uniform over the warp
             const float2* st = stats + p * stats_ld;
-            float mx = -INFINITY;
-            for (int t = lane; t < tiles; t += 32) mx = fmaxf(mx, st[t].x);
+            float* q = chunk_tab ? chunk_tab + p * chunk_ld : nullptr;
+            const float2 first = lane < tiles ? st[lane] : make_float2(-INFINITY, 0.f);
+            float qv[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { const int t = lane + 32 * k; qv[k] = (q && t < n_chunks) ? q[t] : 0.f; }
+            const float zl = zlabel[p];
+            float mx = first.x;
+            for (int t = lane + 32; t < tiles; t += 32) mx = fmaxf(mx, st[t].x);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            double s = 0.0;
-            for (int t = lane; t < tiles; t += 32) {
+            // the tile sums are fp32 sums of fp32 exponentials: rescaling them needs no more than expf
+            double s = (double)first.y * (double)expf(first.x - mx);
+            for (int t = lane + 32; t < tiles; t += 32) {
                 const float2 v = st[t];
-                s += (double)v.y * exp((double)v.x - (double)mx);
+                s += (double)v.y * (double)expf(v.x - mx);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             const double l = (double)mx + log(s);
-            if (chunk_tab) {
-                float* q = chunk_tab + p * chunk_ld;
-                for (int t = lane; t < n_chunks; t += 32) q[t] = expf((float)((double)q[t] - l));
+            if (q) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { const int t = lane + 32 * k; if (t < n_chunks) q[t] = expf((float)((double)qv[k] - l)); }
+                for (int t = lane + 128; t < n_chunks; t += 32) q[t] = expf((float)((double)q[t] - l));
             }
             if (lane == 0) lse[p] = (float)l;
-            term = l - (double)zlabel[p];
+            term = l - (double)zl;
         }
         if (lane == 0) red[row] = term;
     }
@@ -113,12 +122,19 @@ __global__ void rowsums_kernel(const float2* __restrict__ stats, int64_t stats_l
     if (threadIdx.x == 0) block_partials[blockIdx.x] = red[0];
 }
 
-__global__ void loss_final_kernel(const double* __restrict__ block_partials, int nblocks, int accumulate,
-                                  double* __restrict__ loss_out) {
-    // a single thread: a few hundred additions in index order
+__global__ void __launch_bounds__(256)
+loss_final_kernel(const double* __restrict__ block_partials, int nblocks, int accumulate, double* __restrict__ loss_out) {
+    // one block: 256 threads add every 256th partial in index order, then a fixed tree
+    __shared__ double red[256];
     double s = 0.0;
-    for (int i = 0; i < nblocks; ++i) s += block_partials[i];
-    *loss_out = accumulate ? *loss_out + s : s;
+    for (int i = threadIdx.x; i < nblocks; i += 256) s += block_partials[i];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *loss_out = accumulate ? *loss_out + red[0] : red[0];
 }
 
 constexpr int DC_ROWS = 1024;   // patterns per partial row of the delta column sum
@@ -194,7 +210,11 @@ __global__ void dot_final_kernel(const double* __restrict__ parts, int64_t npart
     if (threadIdx.x == 0) *out = red[0];
 }
 
-__global__ void sgd_kernel(float* __restrict__ w, const float* __restrict__ g, int64_t n, float lr) {
+// the same step for several tensors in one launch: blockIdx.y picks the tensor
+__global__ void sgd_multi_kernel(const SgdBatch b, float lr) {
+    float* __restrict__ w = b.w[blockIdx.y];
+    const float* __restrict__ g = b.g[blockIdx.y];
+    const int64_t n = b.n[blockIdx.y];
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         w[i] = fmaf(-lr, g[i], w[i]);
 }
@@ -276,7 +296,7 @@ ulsnn_status_t launch_rowstats(const float2* stats, int64_t stats_ld, int tiles,
         ulsnn::count_launch(2);
         if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
     }
-    loss_final_kernel<<<1, 1, 0, stream>>>(block_partials, nb, accumulate, loss_out);
+    loss_final_kernel<<<1, 256, 0, stream>>>(block_partials, nb, accumulate, loss_out);
     ulsnn::count_launch(2);
     return cuda_ok(cudaGetLastError());
 }
@@ -289,7 +309,7 @@ ulsnn_status_t launch_rowsums(const float2* stats, int64_t stats_ld, int tiles, 
         ulsnn::count_launch(2);
         if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
     }
-    loss_final_kernel<<<1, 1, 0, stream>>>(block_partials, nb, accumulate, loss_out);
+    loss_final_kernel<<<1, 256, 0, stream>>>(block_partials, nb, accumulate, loss_out);
     ulsnn::count_launch(2);
     return cuda_ok(cudaGetLastError());
 }
@@ -352,9 +372,15 @@ ulsnn_status_t launch_dot(int64_t n, const float* x, const float* y, double* out
     return cuda_ok(cudaGetLastError());
 }
 
-ulsnn_status_t launch_sgd(float* w, const float* g, int64_t n, float lr, cudaStream_t stream) {
-    if (n <= 0) return ULSNN_OK;
-    sgd_kernel<<<grid_for(n, 256), 256, 0, stream>>>(w, g, n, lr);
+ulsnn_status_t launch_sgd_multi(const SgdBatch& b, float lr, cudaStream_t stream) {
+    if (b.count <= 0) return ULSNN_OK;
+    if (b.count > SgdBatch::MAX) return ULSNN_ERR_INVALID_ARG;
+    int64_t nmax = 0;
+    for (int i = 0; i < b.count; ++i) if (b.n[i] > nmax) nmax = b.n[i];
+    if (nmax <= 0) return ULSNN_OK;
+    int64_t bx = (nmax + 4 * 256 - 1) / (4 * 256);          // about four elements per thread of the largest tensor
+    if (bx > 148 * 8) bx = 148 * 8;
+    sgd_multi_kernel<<<dim3((unsigned)bx, (unsigned)b.count), 256, 0, stream>>>(b, lr);
     ulsnn::count_launch(2);
     return cuda_ok(cudaGetLastError());
 }
