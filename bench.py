@@ -40,7 +40,7 @@ NOMINAL_TF32_OVER_BF16 = 0.5        # dense TF32 tensor rate is half the BF16 ra
 # DRAM bytes per launch of the dominant kernel from one ncu capture (profiles/tc_gemm_3xtf32_config3.md: measured at
 # 16384 patterns and scaled by the pattern count).  Only reported while the library still is the version the
 # counters were taken on.
-NCU_TRAFFIC = {"library_version": 103, ("config3", "3xtf32", (3203, 481, 65536)): 4 * (301.80838e6 + 22.601216e6)}
+NCU_TRAFFIC = {"library_version": 104, ("config3", "3xtf32", (3203, 481, 65536)): 4 * (301.80838e6 + 22.601216e6)}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

@@ -31,7 +31,7 @@ SIZES5 = [1024, 4096, 4096, 3203]
 N5 = 131072
 
 
-@pytest.mark.parametrize("math_mode", [ul.MATH_3XTF32, ul.MATH_TF32])
+@pytest.mark.parametrize("math_mode", [ul.MATH_3XTF32, ul.MATH_TF32, ul.MATH_BF16])
 def test_config5_sub_batch_against_checker(math_mode):
     # the first 768 patterns of the seeded batch, through a handle sized for the full batch
     n = 768
