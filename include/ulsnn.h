@@ -75,6 +75,9 @@ int ulsnn_version(void);
  * 256-byte aligned and may be reused by the next call on the same stream.
  * Operands that the tensor-core path cannot address with TMA (a base pointer not 16-byte aligned, or a leading
  * dimension that is not a multiple of 4) are computed by the FFMA kernel instead, which is at least as accurate.
+ * ULSNN_MATH_BF16: op(A) and op(B) are first rounded to bfloat16 (round to nearest even) into the workspace, which
+ * therefore is never empty in this mode (two bfloat16 copies with rows padded to 8 elements, then the split-K
+ * partials); any lda / ldb is accepted.  C, alpha and beta stay fp32.  Expect a relative error of about 2e-3.
  * Errors: ULSNN_ERR_INVALID_ARG (nothing launched), ULSNN_ERR_WORKSPACE_TOO_SMALL, ULSNN_ERR_UNSUPPORTED_ARCH, ULSNN_ERR_CUDA.
  */
 ulsnn_status_t ulsnn_sgemm(char transA, char transB, int64_t M, int64_t N, int64_t K, float alpha,

@@ -611,8 +611,9 @@ ulsnn_status_t forward(ulsnn_mlp* h, const float* const* W, const float* const* 
 // ---- 16-bit mode (softmax head).  The batch and the weights are rounded to bfloat16 first; every product then reads
 // and writes bfloat16 (fp32 accumulators, fp32 statistics, loss and gradients).
 ulsnn_status_t forward_bf16(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
-                            const int32_t* labels, int64_t n, bool keep, int accumulate, double* loss_out, cudaStream_t stream) {
+                            const Targets& tg, int64_t n, bool keep, int accumulate, double* loss_out, cudaStream_t stream) {
     const int L = h->L;
+    const int32_t* labels = tg.labels;
     h->n_phases = 0;
     if (h->timing) h->timed_calls++;
     ulsnn_status_t st = launch_to_bf16(X, n, h->sizes[0], ldx, h->Xb, h->ldxb, 1, stream);
@@ -638,23 +639,26 @@ ulsnn_status_t forward_bf16(ulsnn_mlp* h, const float* const* W, const float* co
     d.Ch = keep ? h->Eb : nullptr; d.ldch = h->ldeb;
     d.epi = EPI_LOGITS; d.bias = b[L - 1]; d.labels = labels;
     d.stats = h->stats; d.stats_ld = h->stats_ld; d.zlabel = h->zlabel;
-    d.chunk_max = keep ? h->chunk_tab : nullptr; d.chunk_ld = h->chunk_ld;
+    d.chunk_max = (keep && !tg.T) ? h->chunk_tab : nullptr; d.chunk_ld = h->chunk_ld;
+    if (tg.T) { d.epi = EPI_TANH_SSE; d.T = tg.T; d.ldt = tg.ldt; }     // the output deltas dE/dz go where the exponentials would
     d.splits = 1; d.k_per_split = d.K;
     const int entries = 2 * (int)((d.N + hg_tile_n(d) - 1) / hg_tile_n(d));
     if (entries > h->stats_ld) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
     if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
+    if (tg.T) return launch_rowsums(h->stats, h->stats_ld, entries, n, h->loss_parts, accumulate, loss_out, stream);
     return launch_rowstats(h->stats, h->stats_ld, entries, h->zlabel, n, h->lse, d.chunk_max, h->chunk_ld,
                            (int)(((int64_t)h->sizes[L] + 31) / 32), h->loss_parts, accumulate, loss_out, stream);
 }
 
 ulsnn_status_t gradient_bf16(ulsnn_mlp* h, const float* const* W, const float* const* b, const float* X, int64_t ldx,
-                             const int32_t* labels, int64_t n, int accumulate, float* const* dW, float* const* db,
+                             const Targets& tg, int64_t n, int accumulate, float* const* dW, float* const* db,
                              double* loss_out, cudaStream_t stream) {
     const int L = h->L;
-    ulsnn_status_t st = forward_bf16(h, W, b, X, ldx, labels, n, true, accumulate, loss_out, stream);
+    ulsnn_status_t st = forward_bf16(h, W, b, X, ldx, tg, n, true, accumulate, loss_out, stream);
     if (st != ULSNN_OK) return st;
-    // delta_L = softmax - onehot, in place over the stored exponentials
-    if ((st = launch_delta_bf16(h->Eb, h->ldeb, h->chunk_tab, h->chunk_ld, labels, n, h->sizes[L], stream)) != ULSNN_OK) return st;
+    // softmax head: delta_L = softmax - onehot, in place over the stored exponentials (the squared-error epilogue has
+    // written its deltas already)
+    if (!tg.T && (st = launch_delta_bf16(h->Eb, h->ldeb, h->chunk_tab, h->chunk_ld, tg.labels, n, h->sizes[L], stream)) != ULSNN_OK) return st;
     // delta_l = (1 - H_l*H_l) * (delta_{l+1} W_{l+1})   (H_D of Section 4.2)
     for (int l = L - 1; l >= 1; --l) {
         HalfGemmDesc d{};
@@ -775,9 +779,8 @@ ulsnn_status_t forward_call(ulsnn_mlp_t* h, const float* const* W, const float* 
     if (st != ULSNN_OK) return st;
     if (tg.T && n > 0 && tg.ldt < h->sizes[h->L]) return ULSNN_ERR_INVALID_ARG;
     if ((st = check_arch()) != ULSNN_OK) return st;
-    if (h->math == ULSNN_MATH_BF16 && tg.T) return ULSNN_ERR_INVALID_ARG;     // the 16-bit mode has the softmax head only
     if (n == 0) return launch_zero_f64(loss_out, 1, stream);
-    if (h->math == ULSNN_MATH_BF16) return forward_bf16(h, W, b, X, ldx, tg.labels, n, false, 0, loss_out, stream);
+    if (h->math == ULSNN_MATH_BF16) return forward_bf16(h, W, b, X, ldx, tg, n, false, 0, loss_out, stream);
     return forward(h, W, b, X, ldx, tg, n, false, 0, loss_out, stream);
 }
 
@@ -792,7 +795,6 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
     const bool sse = tg.T != nullptr;
     const int32_t* labels = tg.labels;
     for (int l = 0; l < L; ++l) if (!dW[l] || !db[l]) return ULSNN_ERR_INVALID_ARG;
-    if (h->math == ULSNN_MATH_BF16 && sse) return ULSNN_ERR_INVALID_ARG;
     if ((st = check_arch()) != ULSNN_OK) return st;
     if (n == 0) {
         if (accumulate) return ULSNN_OK;
@@ -802,7 +804,7 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
         }
         return launch_zero_f64(loss_out, 1, stream);
     }
-    if (h->math == ULSNN_MATH_BF16) return gradient_bf16(h, W, b, X, ldx, labels, n, accumulate, dW, db, loss_out, stream);
+    if (h->math == ULSNN_MATH_BF16) return gradient_bf16(h, W, b, X, ldx, tg, n, accumulate, dW, db, loss_out, stream);
     if ((st = forward(h, W, b, X, ldx, tg, n, true, accumulate, loss_out, stream)) != ULSNN_OK) return st;
 
     int64_t colsum_rows = 0;

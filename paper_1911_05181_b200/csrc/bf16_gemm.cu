@@ -295,7 +295,8 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         uint8_t* stg = epi_scratch + ew * (EPI_BUFS * EPI_STAGE_BYTES);
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
         const bool c_vec = ((((uintptr_t)d.C) & 15) == 0) && ((d.ldc & 3) == 0);
-        const bool bias_vec = (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) && ((((uintptr_t)d.bias) & 15) == 0);
+        const bool bias_vec = (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS || EPI == EPI_TANH_SSE) && ((((uintptr_t)d.bias) & 15) == 0);
+        const bool t_vec = (EPI == EPI_TANH_SSE) && ((((uintptr_t)d.T) & 15) == 0) && ((d.ldt & 3) == 0);
         const bool ch_vec = ((((uintptr_t)d.Ch) & 15) == 0) && ((d.ldch & 7) == 0);
         const bool h_vec = (EPI == EPI_TANHP) && ((((uintptr_t)d.Hm) & 15) == 0) && ((d.ldh & 7) == 0);
         uint32_t tile_i = 0, stg_i = 0;
@@ -313,6 +314,18 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             bool have_zl = false;
             int lab = -1;
             if (EPI == EPI_LOGITS && rv) lab = __ldg(d.labels + r);        // asked for before the wait for the products
+            // TANH_SSE: the targets of a 64-column block are brought into L2 one block ahead of their use
+            auto prefetch_targets = [&](int b64) {
+                const int c0 = n0 + b64 * 64;
+                if (EPI == EPI_TANH_SSE && rv && b64 < nblk) {
+                    const float* tp = d.T + r * d.ldt + c0;
+                    const int last = min(63, (int)d.N - c0 - 1);
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(tp));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(tp + (last >> 1)));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(tp + last));
+                }
+            };
+            prefetch_targets(half);
             if (!wait_bar(&ctrl->reg_full[acc], (tile_i >> 1) & 1, ctrl, p.status)) { ok = false; break; }
             tc_fence_after();
 
@@ -332,9 +345,10 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 uint32_t raw[2][32];
                 float bv[2][32];
                 const int nv64 = min(64, (int)d.N - (n0 + blk64 * 64));
+                prefetch_targets(blk64 + 2);
                 tmem_ld32(tmem_base + acc * BN_MAX + (2 * blk64) * 32 + lane_off, raw[0]);
                 if (nv64 > 32) tmem_ld32(tmem_base + acc * BN_MAX + (2 * blk64 + 1) * 32 + lane_off, raw[1]);
-                if (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) {
+                if (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS || EPI == EPI_TANH_SSE) {
 #pragma unroll
                     for (int cc = 0; cc < 2; ++cc) {
                         const int c0 = n0 + (2 * blk64 + cc) * 32;
@@ -382,6 +396,31 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = d.alpha * v[j];
                         }
+                    } else if (EPI == EPI_TANH_SSE) {
+                        // Eqs. 1 and 3: y = tanh(z), E += (y - t)^2, stored value dE/dz = 2 (y - t)(1 - y^2)
+                        float s = 0.f;
+                        if (rv && nvalid > 0) {
+                            const float* tp = d.T + r * d.ldt + c0;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                float4 t4;
+                                if (t_vec && full) t4 = __ldg(reinterpret_cast<const float4*>(tp + j));
+                                else t4 = make_float4(j < nvalid ? __ldg(tp + j) : 0.f, j + 1 < nvalid ? __ldg(tp + j + 1) : 0.f,
+                                                      j + 2 < nvalid ? __ldg(tp + j + 2) : 0.f, j + 3 < nvalid ? __ldg(tp + j + 3) : 0.f);
+                                const float tt[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) {
+                                    const float y = tanh_approx(v[j + t] + bv[cc][j + t]);
+                                    const float e = (j + t < nvalid) ? y - tt[t] : 0.f;
+                                    s += e * e;
+                                    v[j + t] = 2.f * e * (1.f - y * y);
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                        }
+                        run_s += s;
                     } else if (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] += bv[cc][j];
@@ -511,6 +550,7 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 d.stats[r * d.stats_ld + nt * 2 + half] = make_float2(run_m, run_s);
                 if (have_zl) d.zlabel[r] = zl;
             }
+            if (EPI == EPI_TANH_SSE && rv) d.stats[r * d.stats_ld + nt * 2 + half] = make_float2(0.f, run_s);
             if (EPI == EPI_BIAS_TANH && d.ones_cols > 0 && nt == p.tiles_n - 1 && half == 0 && rv) {
                 d.Ch[r * d.ldch + d.N] = __float2bfloat16_rn(1.f);
                 for (int cc = 1; cc < d.ones_cols; ++cc) d.Ch[r * d.ldch + d.N + cc] = __float2bfloat16_rn(0.f);
@@ -730,7 +770,7 @@ ulsnn_status_t hg_gemm_launch(const HalfGemmDesc& d, cudaStream_t stream) {
     const bool b_made = p.b_mn ? make_map16(&mb, d.B, d.N, d.K, d.b_sk, 64, BK, false) : make_map16(&mb, d.B, d.K, d.N, d.b_sn, BK, p.bn / cg, false);
     if (!a_made || !b_made) return ULSNN_ERR_CUDA;
 
-    const bool out16 = d.epi == EPI_BIAS_TANH || d.epi == EPI_LOGITS || d.epi == EPI_TANHP;
+    const bool out16 = d.epi == EPI_BIAS_TANH || d.epi == EPI_LOGITS || d.epi == EPI_TANHP || d.epi == EPI_TANH_SSE;
     if (d.epi == EPI_PARTIAL) {
         p.c_tma = make_store_map32(&mc, d.partials, d.N, d.M, d.ldp, splits) ? 1 : 0;
     } else if (d.epi == EPI_SGEMM) {
@@ -752,6 +792,7 @@ ulsnn_status_t hg_gemm_launch(const HalfGemmDesc& d, cudaStream_t stream) {
         case EPI_LOGITS:    return launch_cg<EPI_LOGITS>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
         case EPI_TANHP:     return launch_cg<EPI_TANHP>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
         case EPI_PARTIAL:   return launch_cg<EPI_PARTIAL>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
+        case EPI_TANH_SSE:  return launch_cg<EPI_TANH_SSE>(cg, ma, mb, mc, p, smem_bytes, grid, stream);
     }
     return ULSNN_ERR_INVALID_ARG;
 }

@@ -65,16 +65,18 @@ struct HalfGemmDesc {
     int64_t M, N, K;
     const __nv_bfloat16* A; int64_t a_sm, a_sk;   // A(i,k) = A[i*a_sm + k*a_sk]  (one of the strides is 1)
     const __nv_bfloat16* B; int64_t b_sk, b_sn;   // B(k,j) = B[k*b_sk + j*b_sn]
-    int epi;                  // EPI_SGEMM, EPI_BIAS_TANH, EPI_LOGITS, EPI_TANHP or EPI_PARTIAL
+    int epi;                  // any Epilogue
     float* C; int64_t ldc;    // SGEMM: fp32 output
     float alpha, beta;
-    __nv_bfloat16* Ch; int64_t ldch;     // BIAS_TANH, LOGITS (may be null: statistics only), TANHP: bfloat16 output
+    __nv_bfloat16* Ch; int64_t ldch;     // BIAS_TANH, LOGITS and TANH_SSE (may be null: statistics only), TANHP: bfloat16 output
     const float* bias;        // [N]  BIAS_TANH, LOGITS
     int ones_cols;            // BIAS_TANH: Ch[:, N] = 1 and Ch[:, N+1 .. N+ones_cols) = 0
     const __nv_bfloat16* Hm; int64_t ldh;        // TANHP
     const int32_t* labels;    // LOGITS
+    const float* T; int64_t ldt;         // TANH_SSE: fp32 targets [M x N]
     float2* stats; int64_t stats_ld;     // LOGITS: stats[row*stats_ld + 2*col_tile + h], h = 0, 1: (max, sum exp(z - max)) over
-                                         // the even (odd) 64-column blocks of the tile; (-inf, 0) when there is none
+                                         // the even (odd) 64-column blocks of the tile; (-inf, 0) when there is none.
+                                         // TANH_SSE: (0, sum (y - t)^2) at the same places
     float* zlabel;
     float* chunk_max; int64_t chunk_ld;  // LOGITS: as in GemmDesc
     int splits; int64_t k_per_split;     // EPI_PARTIAL; k_per_split is a multiple of hg_k_granule()
