@@ -359,7 +359,6 @@ struct ulsnn_mlp {
     float* Wlo[MAX_LAYERS];
     float* D[MAX_LAYERS + 1];
     float* Z;
-    float* D2; float* D2lo;         // delta of the output layer as left behind by the first delta product (pair in 3xTF32)
     float* Zlo;                     // 3xTF32, squared-error head: lo half of the output deltas (Z holds the hi half)
     float2* stats;
     float* lse;
@@ -479,10 +478,6 @@ ulsnn_status_t layout(ulsnn_mlp* h, char* base) {
     }
     h->ldz = round_up((int64_t)h->sizes[L], 4);
     h->Z = (float*)take((size_t)B * h->ldz * sizeof(float));
-    // TF32 mode only: in 3xTF32 mode storing the (hi, lo) tiles slowed the delta product down by more than the
-    // weight-gradient product gained (measured 1.15 -> 1.57 ms against 1.18 -> 0.89 ms at 65536 patterns)
-    h->D2 = (L >= 2 && h->math == ULSNN_MATH_TF32) ? (float*)take((size_t)B * h->ldz * sizeof(float)) : nullptr;
-    h->D2lo = nullptr;
     h->Zlo = (h->math == ULSNN_MATH_3XTF32) ? (float*)take((size_t)B * h->ldz * sizeof(float)) : nullptr;
     h->stats_ld = ((int64_t)h->sizes[L] + 63) / 64;          // enough for any column-tile width >= 64
     h->stats = (float2*)take((size_t)B * h->stats_ld * sizeof(float2));
@@ -808,18 +803,22 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
     if ((st = forward(h, W, b, X, ldx, tg, n, true, accumulate, loss_out, stream)) != ULSNN_OK) return st;
 
     int64_t colsum_rows = 0;
-    bool delta2_kept = false;       // the top delta product ran on the tensor-core engine and left delta_L in D2
     // Deltas of the hidden layers, top down: delta_l = (1 - H_l*H_l) * (delta_{l+1} W_{l+1})   (H_D of Section 4.2).
-    // Softmax head: delta_L is not stored, the kernels form softmax(z) - onehot from the logits as they load them.
-    // Squared-error head: the output epilogue has written delta_L = dE/dz where the logits would be.
+    // Softmax head, 3xTF32 and FFMA modes: delta_L is not stored, the kernels form softmax(z) - onehot from the stored
+    // exponentials as they load them (the operand pass that splits them into TF32 pairs is there anyway).
+    // Softmax head, TF32 mode: a kernel turns the stored exponentials into delta_L in place, so that the two products
+    // that read it need no operand pass at all.
+    // Squared-error head: the output epilogue has written delta_L = dE/dz where the exponentials would be.
+    const bool stored_delta = sse || h->math == ULSNN_MATH_TF32;
+    if (!sse && stored_delta &&
+        (st = launch_delta_inplace(h->Z, h->ldz, h->chunk_tab, h->chunk_ld, labels, n, h->sizes[L], stream)) != ULSNN_OK) return st;
     for (int l = L - 1; l >= 1; --l) {
         GemmDesc d{};
         d.M = n; d.N = h->sizes[l]; d.K = h->sizes[l + 1];
-        if (l + 1 == L && sse) {
+        if (l + 1 == L && stored_delta) {
             d.A = h->Z; d.A_lo = h->Zlo; d.a_sm = h->ldz;
         } else if (l + 1 == L) {
             d.A = h->Z; d.a_sm = h->ldz; d.a_transform = 1; d.scale = h->chunk_tab; d.scale_ld = h->chunk_ld; d.labels = labels; d.a_pattern_is_m = 1;
-            d.delta_out = h->D2; d.delta_out_lo = h->D2lo;      // kept for the weight-gradient product below
         }
         else            { d.A = h->D[l + 1]; d.a_sm = h->ldd[l + 1]; }
         d.a_sk = 1;
@@ -829,7 +828,6 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
         d.epi = EPI_TANHP; d.Hm = h->H[l]; d.Hm_lo = h->Hlo[l]; d.ldh = h->ldh[l];
         d.colsum_part = (l == 1) ? h->colsum_parts : nullptr;
         d.splits = 1; d.k_per_split = d.K;
-        if (l + 1 == L && !sse) delta2_kept = use_tc(d, h->math) && tc_keeps_delta(d, h->math == ULSNN_MATH_3XTF32);
         if (l == 1) colsum_rows = ((n + 127) / 128) * (use_tc(d, h->math) ? tc_colsum_groups() : simt_colsum_groups());
         if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
     }
@@ -840,8 +838,7 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
     for (int w = L - 1; w >= 0; --w) {
         GemmDesc d{};
         d.M = h->sizes[w + 1]; d.N = h->sizes[w] + (w >= 1 ? 1 : 0); d.K = n;
-        if (w + 1 == L && sse) { d.A = h->Z; d.A_lo = h->Zlo; d.a_sk = h->ldz; }
-        else if (w + 1 == L && delta2_kept) { d.A = h->D2; d.A_lo = h->D2lo; d.a_sk = h->ldz; }
+        if (w + 1 == L && stored_delta) { d.A = h->Z; d.A_lo = h->Zlo; d.a_sk = h->ldz; }
         else if (w + 1 == L) { d.A = h->Z; d.a_sk = h->ldz; d.a_transform = 1; d.scale = h->chunk_tab; d.scale_ld = h->chunk_ld; d.labels = labels; d.a_pattern_is_m = 0; }
         else            { d.A = h->D[w + 1]; d.a_sk = h->ldd[w + 1]; }
         d.a_sm = 1;
@@ -860,7 +857,7 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
     // bias gradient of the first layer: column sums of delta_1 (both engines use 128-row tiles)
     if (L >= 2) {
         st = launch_colsum_reduce(h->colsum_parts, colsum_rows, h->sizes[1], accumulate, db[0], stream);
-    } else if (sse) {
+    } else if (stored_delta) {
         st = launch_matrix_colsum(h->Z, h->Zlo, h->ldz, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);
     } else {
         st = launch_delta_colsum(h->Z, h->ldz, h->chunk_tab, h->chunk_ld, labels, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);

@@ -49,10 +49,6 @@ struct GemmDesc {
     int a_transform;
     const float* scale; int64_t scale_ld;
     int a_pattern_is_m;       // 1: the M index of A is the pattern (K is the class); 0: K is the pattern
-    // Optional copy of the transformed operand (tensor-core engine, a_pattern_is_m == 1 only): delta = softmax - onehot
-    // is also written to delta_out (and, in 3xTF32 mode, as the pair tf32_rn(delta) -> delta_out, remainder ->
-    // delta_out_lo), [patterns x classes] with the row stride of A, for the product that needs it next.
-    float* delta_out; float* delta_out_lo;
     // split-K (EPI_PARTIAL): slice s covers k in [s*k_per_split, min(K, (s+1)*k_per_split))
     int splits; int64_t k_per_split;
     float* partials; int64_t ldp;        // partials[(s*M + i)*ldp + j]
@@ -93,8 +89,6 @@ int simt_tile_n();
 // tcgen05 engine (tc_gemm.cu).  tc_gemm_supported: can TMA address these operands (16-byte aligned bases, leading
 // dimensions that are multiples of 4 floats)?  tc_tile_n: the column-tile width it will use for this product.
 bool tc_gemm_supported(const GemmDesc& d);
-// will the tensor-core engine leave the transformed operand in d.delta_out (see GemmDesc)?
-bool tc_keeps_delta(const GemmDesc& d, bool three_x);
 int tc_tile_m(const GemmDesc& d);
 int tc_tile_n(const GemmDesc& d);
 // how many tiles each engine works on at a time (CTAs, or CTA pairs): what a split-K plan has to fill
@@ -151,6 +145,10 @@ ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* sca
                                    int64_t n, int64_t n_classes, float* parts, int accumulate, float* out,
                                    cudaStream_t stream);
 int delta_colsum_tiles(int64_t n);
+// in place: stored exponentials Z [n x ldz] (ldz a multiple of 4, 16-byte aligned) -> Z * scale[pattern][class/32] - onehot,
+// zero in the row padding
+ulsnn_status_t launch_delta_inplace(float* Z, int64_t ldz, const float* scale, int64_t scale_ld, const int32_t* labels,
+                                    int64_t n, int64_t n_classes, cudaStream_t stream);
 // hi[i] = tf32_rn(x[i]), lo[i] = tf32_rn(x[i] - hi[i])   (round to nearest, ties away from zero, 10 mantissa bits)
 ulsnn_status_t launch_split_hilo(const float* x, int64_t n, float* hi, float* lo, cudaStream_t stream);
 // out = a*x + b*y (out may alias x or y); *out = sum_i x[i]*y[i] in double, blocks of 1024 elements in index order

@@ -160,6 +160,27 @@ __global__ void delta_colsum_kernel(const float* __restrict__ Z, int64_t ldz, co
     parts[(int64_t)blockIdx.y * n_classes + j] = s;
 }
 
+// In place: Z[p][j] (= exp(z - m) as the LOGITS epilogue left it) -> Z[p][j] * scale[p][j/32] - [label_p == j], zero in
+// the row padding.  One thread per four elements (ldz is a multiple of 4), which lie in one 32-class chunk.
+__global__ void delta_inplace_kernel(float* __restrict__ Z, int64_t ldz, const float* __restrict__ scale, int64_t scale_ld,
+                                     const int32_t* __restrict__ labels, int64_t n, int n_classes) {
+    const int64_t groups = ldz >> 2;
+    const int64_t total = n * groups;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t pat = e / groups;
+        const int j0 = (int)(e - pat * groups) << 2;
+        float4* ptr = reinterpret_cast<float4*>(Z + pat * ldz + j0);
+        float4 v = *ptr;
+        const float f = (j0 < n_classes) ? __ldg(scale + pat * scale_ld + (j0 >> 5)) : 0.f;
+        const int lab = __ldg(labels + pat);
+        v.x = (j0 + 0 < n_classes) ? fmaf(v.x, f, j0 + 0 == lab ? -1.f : 0.f) : 0.f;
+        v.y = (j0 + 1 < n_classes) ? fmaf(v.y, f, j0 + 1 == lab ? -1.f : 0.f) : 0.f;
+        v.z = (j0 + 2 < n_classes) ? fmaf(v.z, f, j0 + 2 == lab ? -1.f : 0.f) : 0.f;
+        v.w = (j0 + 3 < n_classes) ? fmaf(v.w, f, j0 + 3 == lab ? -1.f : 0.f) : 0.f;
+        *ptr = v;
+    }
+}
+
 __device__ __forceinline__ float round_tf32(float x) {
     return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
 }
@@ -341,6 +362,15 @@ ulsnn_status_t launch_delta_colsum(const float* Z, int64_t ldz, const float* sca
         if (cudaGetLastError() != cudaSuccess) return ULSNN_ERR_CUDA;
     }
     return launch_colsum_reduce(parts, tiles, n_classes, accumulate, out, stream);
+}
+
+ulsnn_status_t launch_delta_inplace(float* Z, int64_t ldz, const float* scale, int64_t scale_ld, const int32_t* labels,
+                                    int64_t n, int64_t n_classes, cudaStream_t stream) {
+    if (n <= 0) return ULSNN_OK;
+    if ((ldz & 3) != 0 || (((uintptr_t)Z) & 15) != 0) return ULSNN_ERR_INVALID_ARG;
+    delta_inplace_kernel<<<grid_for(n * (ldz >> 2), 256), 256, 0, stream>>>(Z, ldz, scale, scale_ld, labels, n, (int)n_classes);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
 }
 
 ulsnn_status_t launch_split_hilo(const float* x, int64_t n, float* hi, float* lo, cudaStream_t stream) {

@@ -3,8 +3,7 @@
 // and the fused epilogues.
 //
 // One persistent CTA per SM, 14 warps with fixed roles:
-//   warp 0      TMA producer      global -> swizzled shared-memory stages (cp.async.bulk.tensor, no multicast);
-//                                 also stores transformed A stages back to global memory when deltas are kept
+//   warp 0      TMA producer      global -> swizzled shared-memory stages (cp.async.bulk.tensor, no multicast)
 //   warp 1      product issuer    all lanes run the loop, an elected lane issues tcgen05.mma.kind::tf32 and the
 //                                 commits (in the second CTA of a pair: relays "stage ready" to the first)
 //   warps 2-5   epilogue          tcgen05.ld of the 128 x BN fp32 accumulator (one row per thread), fused math, then
@@ -74,7 +73,6 @@ struct TcParams {
     int three_x, a_mn, b_mn, split_pass;
     int a_pre, b_pre;       // 3xTF32: the operand arrives as a stored (hi, lo) pair, no operand pass for it
     int c_pair;             // BIAS_TANH: the output is written as a (hi, lo) pair
-    int d_out;              // the transformed A tiles (deltas) of the first column tile are also stored to global memory
     int chunk_blocks;       // k-blocks accumulated on one TMEM accumulator before it is added into the tile total
     int fast_math;          // TF32 mode: approximate exp
     int c_tma;              // the output (C or the split-K partials) is written with TMA stores
@@ -195,8 +193,7 @@ template <int EPI, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_a_lo, const __grid_constant__ CUtensorMap map_b_lo,
-               const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c_lo,
-               const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_d_lo, const TcParams p) {
+               const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c_lo, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128B swizzle pattern repeats every 8 rows of 128 bytes
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -248,23 +245,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------------ TMA producer
         RingPos rp{0, 0};
         bool ok = true;
-        // Deltas kept for a later product (p.d_out): the transformed A tile of a stage (and its lo part) is stored
-        // from shared memory with TMA, for the first column tile of every row block.  This warp does it two stages
-        // behind its loads -- by then the operand pass of that stage is normally done -- and before it refills a
-        // stage it makes sure that the store which read the stage's previous contents has finished reading.
-        struct Kept { int s; uint32_t phase; int k0, m0; bool store; };
-        Kept h1{-1, 0, 0, 0, false}, h2{-1, 0, 0, 0, false};
-        auto keep = [&](const Kept& h) {
-            if (h.s < 0 || !h.store || !ok) return;
-            if (!wait_bar_warp(&ctrl->ready[h.s], h.phase, ctrl, p.status)) { ok = false; return; }
-            if (elect_one()) {
-                const uint32_t sa = smem_u32(stage_base + (size_t)h.s * p.stage_bytes);
-                tma_store_2d(&map_d, sa + off_a_hi, h.k0, h.m0);
-                if (p.three_x) tma_store_2d(&map_d_lo, sa + off_a_lo, h.k0, h.m0);
-                bulk_commit();
-            }
-            __syncwarp();
-        };
         for (int u = first_unit; u < p.units && ok; u += unit_step) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
             int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
@@ -279,15 +259,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int k0 = (int)kbeg;
             for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
                 const int s = rp.stage;
-                if (p.d_out) {
-                    keep(h2);
-                    if (!ok) break;
-                    // every store but the one just issued has read its stage: stage s may be refilled
-                    if (elect_one()) { if (h2.s >= 0 && h2.store) bulk_wait_read_1(); else bulk_wait_read_0(); }
-                    __syncwarp();
-                    h2 = h1;
-                    h1 = Kept{s, rp.phase, k0, m0, nt == 0};
-                }
                 if (!wait_bar_warp(&ctrl->empty[s], rp.phase ^ 1, ctrl, p.status)) { ok = false; break; }
                 rp.advance(p.stages);
                 const uint32_t bar = smem_u32(&ctrl->full[s]);
@@ -332,11 +303,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 __syncwarp();
             }
-        }
-        if (p.d_out) {
-            keep(h2);
-            keep(h1);
-            if (elect_one()) bulk_wait_all();
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
@@ -904,7 +870,7 @@ int* status_ptr() {
     return ptr;
 }
 
-struct Maps { CUtensorMap a, b, a_lo, b_lo, c, c_lo, d, d_lo; };
+struct Maps { CUtensorMap a, b, a_lo, b_lo, c, c_lo; };
 
 template <int EPI, int CG>
 ulsnn_status_t launch(const Maps& m, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
@@ -924,7 +890,7 @@ ulsnn_status_t launch(const Maps& m, const TcParams& p, int smem_bytes, int grid
     attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG>, m.a, m.b, m.a_lo, m.b_lo, m.c, m.c_lo, m.d, m.d_lo, p);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG>, m.a, m.b, m.a_lo, m.b_lo, m.c, m.c_lo, p);
     count_launch(1);
     return cuda_ok(e == cudaSuccess ? cudaGetLastError() : e);
 }
@@ -968,11 +934,6 @@ bool tc_gemm_supported(const GemmDesc& d) {
     // logits as the A operand: either [pattern x class] read K-major or its transpose read MN-major
     if (d.a_transform && (a_k != (d.a_pattern_is_m != 0))) return false;
     return true;
-}
-
-bool tc_keeps_delta(const GemmDesc& d, bool three_x) {
-    return d.a_transform && d.delta_out && d.a_sk == 1 && BK == 32 && (((uintptr_t)d.delta_out) & 15) == 0 &&
-           (!three_x || (d.delta_out_lo && (((uintptr_t)d.delta_out_lo) & 15) == 0));
 }
 
 ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stream) {
@@ -1021,12 +982,6 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     if (p.a_pre && !map_of_a(&m.a_lo, d.A_lo)) return ULSNN_ERR_CUDA;
     if (p.b_pre && !map_of_b(&m.b_lo, d.B_lo)) return ULSNN_ERR_CUDA;
     p.c_pair = ((d.epi == EPI_BIAS_TANH || d.epi == EPI_TANH_SSE) && d.C_lo) ? 1 : 0;
-    // deltas kept for a later product: the transformed K-major A tile in shared memory is exactly one TMA box
-    if (tc_keeps_delta(d, three_x)) {
-        p.d_out = make_map(&m.d, d.delta_out, d.K, d.M, d.a_sm, BK, BM, false) &&
-                  (!three_x || make_map(&m.d_lo, d.delta_out_lo, d.K, d.M, d.a_sm, BK, BM, false)) ? 1 : 0;
-    }
-
     // the output goes through TMA stores when its rows are 16-byte aligned; otherwise the epilogue stores directly
     if (d.epi == EPI_PARTIAL) {
         p.c_tma = make_store_map(&m.c, d.partials, d.N, d.M, d.ldp, splits) ? 1 : 0;
