@@ -5,13 +5,16 @@
 // the epilogues write are bfloat16 again, so that every later product reads half the bytes.
 //
 // One persistent CTA per SM, 10 warps:
-//   warp 0      TMA producer      global -> 128B-swizzled shared-memory stages (no multicast)
-//   warp 1      product issuer    an elected lane issues the products and commits (second CTA of a pair: relays
-//                                 "stage landed" to the first)
+//   warps 0,10  TMA producers     global -> 128B-swizzled shared-memory stages (no multicast); warp 0 fetches the A
+//                                 tiles and warp 10 the B tiles: a thread gets its next copy accepted only some
+//                                 hundred nanoseconds after the previous one, so two issuers nearly double the rate
+//   warp 1      product issuer    an elected lane issues the products and commits (idle in the second CTA of a pair)
 //   warps 2-9   epilogue          two warps per TMEM lane quarter, each taking every other 64-column block of the
 //                                 128 x BN fp32 accumulator: fused math, then blocks staged in swizzled shared
 //                                 memory and written with TMA stores
-// Tiles are 128 x BN, or 256 x BN by the two CTAs of a cluster (cta_group::2), BN <= 256; TMEM holds two
+// Tiles are 128 x BN, or 256 x BN by the two CTAs of a cluster (cta_group::2), BN <= 256: each CTA fetches its own
+// halves of the operands, and both count the landed bytes on the first CTA's barrier (cta_group::2 form of the TMA
+// load), so that the issuer there waits on one barrier for the whole stage.  TMEM holds two
 // accumulators, so the epilogue of a tile overlaps the products of the next.  There is no operand pass: every
 // byte the tensor core reads arrived by TMA.
 // K-major operands: rows of 64 elements (128 bytes), 128B swizzle.  MN-major operands: boxes of 64 (M or N) x 64
@@ -33,14 +36,15 @@ constexpr int BN_MAX = 256;
 constexpr int BK = 64;                  // elements of K per stage: a K-major tile row is 128 bytes
 constexpr int UMMA_K = 16;              // K of one tcgen05.mma.kind::f16
 constexpr int NUM_EPI_WARPS = 8;
-constexpr int NUM_WARPS = 2 + NUM_EPI_WARPS;
+constexpr int PROD_B_WARP = 2 + NUM_EPI_WARPS;      // second producer warp
+constexpr int NUM_WARPS = 3 + NUM_EPI_WARPS;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 8;
 constexpr int NUM_SMS = 148;
 constexpr int A_TILE_BYTES = BM * BK * 2;
 constexpr int SMEM_BUDGET = 227 * 1024;
 constexpr int EPI_STAGE_BYTES = 32 * 128;           // one block of 32 rows x 128 bytes (64 bf16 or 32 fp32), 128B-swizzled
-constexpr int EPI_BUFS = 2;
+constexpr int EPI_BUFS = 1;
 constexpr int EPI_SCRATCH_BYTES = NUM_EPI_WARPS * EPI_BUFS * EPI_STAGE_BYTES;
 constexpr int CTRL_BYTES = 1024;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 3000000000ull;
@@ -55,12 +59,10 @@ struct HgParams {
 };
 
 struct Ctrl {
-    uint64_t full[MAX_STAGES];      // TMA bytes landed
-    uint64_t ready[MAX_STAGES];     // CTA 0 of a pair: the other CTA's stage has landed too
+    uint64_t full[MAX_STAGES];      // TMA bytes landed (CTA 0 of a pair: the bytes of both CTAs)
     uint64_t empty[MAX_STAGES];     // products that read the stage have completed
     uint64_t reg_full[2];           // the products of the tile in TMEM region r have completed
     uint64_t reg_free[2];           // the epilogue warps have read region r
-    uint64_t relay_sink[MAX_STAGES];
     uint64_t free_sink[2][NUM_EPI_WARPS];
     uint32_t tmem_base;
     volatile int abort;
@@ -160,8 +162,7 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&ctrl->full[s]), 1);
-            mbar_init(smem_u32(&ctrl->ready[s]), 1);        // CTA 0 of a pair: the issuing warp's own arrival posts the 8 bytes CTA 1 sends
+            mbar_init(smem_u32(&ctrl->full[s]), 2);         // one arrival (with its byte count) from each producer warp
             mbar_init(smem_u32(&ctrl->empty[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -181,8 +182,9 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const uint32_t tmem_base = ctrl->tmem_base;
     const int off_a = 0, off_b = A_TILE_BYTES;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+    if (warp == 0 || warp == PROD_B_WARP) {
+        // ------------------------------------------------------------------ TMA producers (A tiles / B tiles)
+        const bool do_a = warp == 0;
         RingPos rp{0, 0};
         bool ok = true;
         for (int u = first_unit; u < p.units && ok; u += unit_step) {
@@ -192,30 +194,38 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int m0 = (mt * CG + rank) * BM, n0 = nt * p.bn + rank * b_cols;
             const int b_boxes = b_cols >> 6;        // MN-major B: boxes of 64 columns, only those the products read
             const uint32_t b_bytes = (uint32_t)(p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes);
-            const uint32_t tx_bytes = (uint32_t)A_TILE_BYTES + b_bytes;
             int k0 = (int)kbeg;
             for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
                 const int s = rp.stage;
                 if (!wait_bar_warp(&ctrl->empty[s], rp.phase ^ 1, ctrl, p.status)) { ok = false; break; }
                 rp.advance(p.stages);
-                const uint32_t bar = smem_u32(&ctrl->full[s]);
+                const uint32_t bar_local = smem_u32(&ctrl->full[s]);
+                const uint32_t bar = (CG == 2) ? addr_in_rank0(bar_local) : bar_local;
                 const uint32_t sa = smem_u32(stage_base + (size_t)s * p.stage_bytes + off_a);
                 const uint32_t sb = sa + off_b;
+                auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+                    if constexpr (CG == 2) tma_load_2d_pair(dst, map, x, y, bar); else tma_load_2d(dst, map, x, y, bar);
+                };
                 if (elect_one()) {
-                    mbar_expect_tx(bar, tx_bytes);
-                    if (!p.a_mn) {
-                        tma_load_2d(sa, &map_a, k0, m0, bar);                       // box {64 k, 128 rows}
-                    } else {
+                    // CTA 0 announces the bytes of both CTAs of the pair (they fetch the same amounts)
+                    if (do_a) {
+                        if (rank == 0) mbar_expect_tx(bar_local, (uint32_t)A_TILE_BYTES * CG);
+                        if (!p.a_mn) {
+                            load(sa, &map_a, k0, m0);                                   // box {64 k, 128 rows}
+                        } else {
 #pragma unroll
-                        for (int g = 0; g < BM / 64; ++g)                           // boxes {64 m, 64 k}
-                            tma_load_2d(sa + g * (BK * 128), &map_a, m0 + 64 * g, k0, bar);
-                    }
-                    if (!p.b_mn) {
-                        tma_load_2d(sb, &map_b, k0, n0, bar);                       // box {64 k, bn/CG rows}
+                            for (int g = 0; g < BM / 64; ++g)                           // boxes {64 m, 64 k}
+                                load(sa + g * (BK * 128), &map_a, m0 + 64 * g, k0);
+                        }
                     } else {
+                        if (rank == 0) mbar_expect_tx(bar_local, b_bytes * CG);
+                        if (!p.b_mn) {
+                            load(sb, &map_b, k0, n0);                                   // box {64 k, bn/CG rows}
+                        } else {
 #pragma unroll
-                        for (int g = 0; g < BN_MAX / 64; ++g)
-                            if (g < b_boxes) tma_load_2d(sb + g * (BK * 128), &map_b, n0 + 64 * g, k0, bar);
+                            for (int g = 0; g < BN_MAX / 64; ++g)
+                                if (g < b_boxes) load(sb + g * (BK * 128), &map_b, n0 + 64 * g, k0);
+                        }
                     }
                 }
                 __syncwarp();
@@ -253,10 +263,6 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 for (int kb = 0; kb < nkb; ++kb) {
                     const int s = rp.stage;
                     if (!wait_bar_warp(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
-                    if (CG == 2) {
-                        if (elect_one()) mbar_expect_tx(smem_u32(&ctrl->ready[s]), 8);
-                        if (!wait_bar_warp(&ctrl->ready[s], rp.phase, ctrl, p.status)) { ok = false; break; }
-                    }
                     rp.advance(p.stages);
                     tc_fence_after();
                     const uint32_t soff = (uint32_t)s * stage_inc;
@@ -272,22 +278,7 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if (ok) umma_commit<CG>(smem_u32(&ctrl->reg_full[reg]));
             }
         }
-        if (CG == 2 && rank == 1) {
-            RingPos rp{0, 0};
-            bool ok = true;
-            for (int u = first_unit; u < p.units && ok; u += unit_step) {
-                int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-                int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
-                for (int kb = 0; kb < nkb; ++kb) {
-                    const int s = rp.stage;
-                    if (!wait_bar_warp(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
-                    rp.advance(p.stages);
-                    if (lane == 0) signal_rank0(smem_u32(&ctrl->relay_sink[s]), smem_u32(&ctrl->ready[s]));
-                    __syncwarp();
-                }
-            }
-        }
-    } else {
+    } else if (warp < 2 + NUM_EPI_WARPS) {
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                         // TMEM lane quarter this warp may read
         const int ew = warp - 2;                        // 0..7
