@@ -2,8 +2,9 @@
 // the error-compensated 3xTF32 mode (operands as TF32 hi/lo pairs, split on chip or loaded as stored pairs),
 // and the fused epilogues.
 //
-// One persistent CTA per SM, 14 warps with fixed roles:
-//   warp 0      TMA producer      global -> swizzled shared-memory stages (cp.async.bulk.tensor, no multicast)
+// One persistent CTA per SM, 16 warps with fixed roles:
+//   warps 0,14,15 TMA producers   global -> swizzled shared-memory stages (cp.async.bulk.tensor, no multicast):
+//                                 warp 0 the A tiles, warp 14 the B tiles, warp 15 the lo halves of stored pairs
 //   warp 1      product issuer    all lanes run the loop, an elected lane issues tcgen05.mma.kind::tf32 and the
 //                                 commits (in the second CTA of a pair: relays "stage ready" to the first)
 //   warps 2-5   epilogue          tcgen05.ld of the 128 x BN fp32 accumulator (one row per thread), fused math, then
@@ -50,7 +51,11 @@ constexpr int CPR = ROW_BYTES / 16;     // 16-byte pieces per K-major row
 constexpr int UMMA_K = 8;               // K of one tcgen05.mma.kind::tf32
 constexpr int NUM_EPI_WARPS = 4;
 constexpr int NUM_SPLIT_WARPS = 8;
-constexpr int NUM_WARPS = 2 + NUM_EPI_WARPS + NUM_SPLIT_WARPS;
+constexpr int NUM_PRODUCERS = 3;         // warp 0 and the last two warps: a thread gets its next TMA copy accepted only
+                                        // some hundred nanoseconds after the previous one, so the copies of a stage
+                                        // are spread over three issuing threads
+constexpr int FIRST_EXTRA_PRODUCER = 2 + NUM_EPI_WARPS + NUM_SPLIT_WARPS;
+constexpr int NUM_WARPS = FIRST_EXTRA_PRODUCER + NUM_PRODUCERS - 1;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 12;
 constexpr int NUM_SMS = 148;               // B200; fixes the tile schedule (and with it every summation order)
@@ -76,6 +81,9 @@ struct TcParams {
     int chunk_blocks;       // k-blocks accumulated on one TMEM accumulator before it is added into the tile total
     int fast_math;          // TF32 mode: approximate exp
     int c_tma;              // the output (C or the split-K partials) is written with TMA stores
+    int producers;          // producer warps that have something to fetch (2 or 3)
+    int direct;             // CTA pairs without an operand pass: both CTAs count their landed bytes on CTA 0's `full`
+                            // barriers (cta_group::2 loads), nothing is relayed
     int64_t n_patterns, n_classes;      // bounds of the logits operand when a_transform
     int* status;
 };
@@ -213,9 +221,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&ctrl->full[s]), 1);
+            mbar_init(smem_u32(&ctrl->full[s]), p.producers);      // one arrival (with its byte count) per producer warp at work
             // CTA 0: its own operand-pass warps plus one arrival relayed from CTA 1; CTA 1: its operand-pass warps
-            const int ready_count = (p.split_pass ? NUM_SPLIT_WARPS : 0) + ((CG == 2 && rank == 0) ? 1 : 0);
+            const int ready_count = (p.split_pass ? NUM_SPLIT_WARPS : 0) + ((CG == 2 && rank == 0 && !p.direct) ? 1 : 0);
             mbar_init(smem_u32(&ctrl->ready[s]), ready_count > 0 ? ready_count : 1);      // unused when nothing arrives on it
             mbar_init(smem_u32(&ctrl->empty[s]), 1);
         }
@@ -241,10 +249,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int off_a_hi = 0, off_b_hi = A_TILE_BYTES;
     const int off_a_lo = A_TILE_BYTES + p.b_tile_bytes, off_b_lo = 2 * A_TILE_BYTES + p.b_tile_bytes;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+    if (warp == 0 || warp >= FIRST_EXTRA_PRODUCER) {
+        // ------------------------------------------------------------------ TMA producers
+        // role 0: the A tiles (and their lo halves when both operands are stored pairs); role 1: the B tiles;
+        // role 2: the lo halves of B, or those of A when only A is a stored pair
+        const int role = warp == 0 ? 0 : warp - FIRST_EXTRA_PRODUCER + 1;
+        const bool get_a = role == 0, get_b = role == 1;
+        const bool get_a_lo = p.a_pre && (p.b_pre ? role == 0 : role == 2), get_b_lo = p.b_pre && role == 2;
         RingPos rp{0, 0};
-        bool ok = true;
+        bool ok = get_a || get_b || get_a_lo || get_b_lo;
         for (int u = first_unit; u < p.units && ok; u += unit_step) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
             int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
@@ -255,51 +268,45 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // a box per 32 columns, and only the boxes the products read are fetched
             const int b_boxes = b_cols >> 5;
             const uint32_t b_bytes = (uint32_t)(p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes);
-            const uint32_t tx_bytes = (uint32_t)A_TILE_BYTES * (p.a_pre ? 2u : 1u) + b_bytes * (p.b_pre ? 2u : 1u);
+            // what this warp fetches per stage; with direct counting CTA 0 announces the bytes of both CTAs
+            const uint32_t tx_bytes = ((get_a ? (uint32_t)A_TILE_BYTES : 0u) + (get_a_lo ? (uint32_t)A_TILE_BYTES : 0u) +
+                                       (get_b ? b_bytes : 0u) + (get_b_lo ? b_bytes : 0u)) * (p.direct ? (uint32_t)CG : 1u);
             int k0 = (int)kbeg;
             for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
                 const int s = rp.stage;
                 if (!wait_bar_warp(&ctrl->empty[s], rp.phase ^ 1, ctrl, p.status)) { ok = false; break; }
                 rp.advance(p.stages);
-                const uint32_t bar = smem_u32(&ctrl->full[s]);
+                const uint32_t bar_local = smem_u32(&ctrl->full[s]);
+                const uint32_t bar = (CG == 2 && p.direct) ? addr_in_rank0(bar_local) : bar_local;
                 const uint32_t sa = smem_u32(stage_base + (size_t)s * p.stage_bytes + off_a_hi);
                 const uint32_t sb = sa + off_b_hi;
-                if (elect_one()) {
-                    mbar_expect_tx(bar, tx_bytes);
+                auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+                    if (CG == 2 && p.direct) tma_load_2d_pair(dst, map, x, y, bar); else tma_load_2d(dst, map, x, y, bar);
+                };
+                auto load_a = [&](uint32_t dst, const CUtensorMap* map) {
                     if (!p.a_mn) {
-                        tma_load_2d(sa, &map_a, k0, m0, bar);                       // box {BK k, 128 rows}
+                        load(dst, map, k0, m0);                                     // box {BK k, 128 rows}
                     } else {
 #pragma unroll
-                        for (int g = 0; g < BM / 32; ++g)                           // boxes {32 m, BK k}
-                            tma_load_2d(sa + g * (BK * 128), &map_a, m0 + 32 * g, k0, bar);
+                        for (int g = 0; g < BM / 32; ++g) load(dst + g * (BK * 128), map, m0 + 32 * g, k0);    // boxes {32 m, BK k}
                     }
+                };
+                auto load_b = [&](uint32_t dst, const CUtensorMap* map) {
                     if (!p.b_mn) {
-                        tma_load_2d(sb, &map_b, k0, n0, bar);                       // box {BK k, bn/CG rows}
+                        load(dst, map, k0, n0);                                     // box {BK k, bn/CG rows}
                     } else {
 #pragma unroll
                         for (int g = 0; g < BN_MAX / 32; ++g)
-                            if (g < b_boxes) tma_load_2d(sb + g * (BK * 128), &map_b, n0 + 32 * g, k0, bar);
+                            if (g < b_boxes) load(dst + g * (BK * 128), map, n0 + 32 * g, k0);
                     }
+                };
+                if (elect_one()) {
+                    if (!p.direct || rank == 0) mbar_expect_tx(bar_local, tx_bytes);
+                    if (get_a) load_a(sa, &map_a);
+                    if (get_b) load_b(sb, &map_b);
                     // operands stored as (hi, lo) pairs: the lo tiles land beside the hi tiles
-                    if (p.a_pre) {
-                        const uint32_t sal = sa + off_a_lo;
-                        if (!p.a_mn) {
-                            tma_load_2d(sal, &map_a_lo, k0, m0, bar);
-                        } else {
-#pragma unroll
-                            for (int g = 0; g < BM / 32; ++g) tma_load_2d(sal + g * (BK * 128), &map_a_lo, m0 + 32 * g, k0, bar);
-                        }
-                    }
-                    if (p.b_pre) {
-                        const uint32_t sbl = sa + off_b_lo;
-                        if (!p.b_mn) {
-                            tma_load_2d(sbl, &map_b_lo, k0, n0, bar);
-                        } else {
-#pragma unroll
-                            for (int g = 0; g < BN_MAX / 32; ++g)
-                                if (g < b_boxes) tma_load_2d(sbl + g * (BK * 128), &map_b_lo, n0 + 32 * g, k0, bar);
-                        }
-                    }
+                    if (get_a_lo) load_a(sa + off_a_lo, &map_a_lo);
+                    if (get_b_lo) load_b(sa + off_b_lo, &map_b_lo);
                 }
                 __syncwarp();
             }
@@ -351,9 +358,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const int s = rp.stage;
                     if (!p.split_pass && !wait_bar_warp(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
                     // CTA 1's signal for this stage completes 8 transaction bytes on `ready`; posting the expectation is
-                    // this warp's own arrival on it
-                    if (CG == 2 && elect_one()) mbar_expect_tx(smem_u32(&ctrl->ready[s]), 8);
-                    if ((p.split_pass || CG == 2) && !wait_bar_warp(&ctrl->ready[s], rp.phase, ctrl, p.status)) { ok = false; break; }
+                    // this warp's own arrival on it (not needed when CTA 1's bytes are counted on `full` directly)
+                    const bool relayed = CG == 2 && !p.direct;
+                    if (relayed && elect_one()) mbar_expect_tx(smem_u32(&ctrl->ready[s]), 8);
+                    if ((p.split_pass || relayed) && !wait_bar_warp(&ctrl->ready[s], rp.phase, ctrl, p.status)) { ok = false; break; }
                     rp.advance(p.stages);
                     tc_fence_after();
                     const uint32_t soff = (uint32_t)s * stage_inc;
@@ -383,7 +391,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
             }
         }
-        if (CG == 2 && rank == 1) {
+        if (CG == 2 && rank == 1 && !p.direct) {
             // CTA 1 issues nothing: this warp tells CTA 0 when a stage of CTA 1 is ready for the products
             RingPos rp{0, 0};
             bool ok = true;
@@ -955,6 +963,8 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.a_pre = (three_x && d.A_lo && !d.a_transform) ? 1 : 0;
     p.b_pre = (three_x && d.B_lo) ? 1 : 0;
     p.split_pass = (d.a_transform || (three_x && !(p.a_pre && p.b_pre))) ? 1 : 0;
+    p.producers = 2 + ((p.a_pre || p.b_pre) ? 1 : 0);
+    p.direct = (cg == 2 && !p.split_pass) ? 1 : 0;
     p.fast_math = three_x ? 0 : 1;
     p.chunk_blocks = three_x ? 256 / BK : (1 << 30);       // 256 elements of K per accumulator in the accurate mode
     p.b_tile_bytes = (p.bn / cg) * ROW_BYTES;
