@@ -3,7 +3,7 @@ search made of an exponential step-size scheme that brackets the minimum by the 
 derivative (estimated on a subset of the patterns) and one quadratic interpolation of the error.
 
 TEST INFRASTRUCTURE ONLY, float64 numpy, independent of the CUDA path.  The paper gives the ingredients but no
-constants and no order of evaluation; the reading taken here (listed in the design doc) is:
+constants and no order of evaluation; the reading taken here is:
 
   direction   d_0 = -g_0;  d_k = -g_k + beta_k d_{k-1},  beta_k = max(0, g_k.(g_k - g_{k-1}) / g_{k-1}.g_{k-1})
   bracketing  slope(a) = grad_subset(w + a d) . d.  From a_0, while slope(a_j) < 0: a_{j+1} = 2 a_j (at most
