@@ -142,3 +142,17 @@ def test_squared_error_head_rejects_bad_arguments_on_the_host():
     assert lib.ulsnn_mlp_gradient_sse(h, ptrs, ptrs, fake, 8, fake, 3, 17, 0, ptrs, ptrs, fake, None) == ul.ERR_INVALID_ARG   # n > max
     assert lib.ulsnn_mlp_gradient_sse(h, ptrs, ptrs, fake, 8, fake, 3, 4, 0, None, ptrs, fake, None) == ul.ERR_INVALID_ARG
     lib.ulsnn_mlp_destroy(h)
+
+
+def test_sixteen_bit_mode_workspaces():
+    # the bf16 SGEMM always needs room for its two operand copies (rows padded to 8 elements), split or not
+    b = ul.sgemm_workspace_bytes("N", "N", 4096, 4096, 4096, ul.MATH_BF16)
+    assert b == 2 * 4096 * 4096 * 2
+    b = ul.sgemm_workspace_bytes("N", "T", 100, 50, 30, ul.MATH_BF16)
+    assert b % 256 == 0 and b >= 100 * 32 * 2 + 50 * 32 * 2
+    # the network keeps bfloat16 activations, exponentials and deltas: well under the fp32 modes' workspace
+    half = ul.mlp_workspace_bytes([400, 480, 3203], ul.MATH_BF16, 65536)
+    full = ul.mlp_workspace_bytes([400, 480, 3203], ul.MATH_TF32, 65536)
+    assert 65536 * 3208 * 2 < half < 0.7 * full
+    with pytest.raises(ul.UlsnnError):
+        ul.mlp_workspace_bytes([400, 480, 3203], 4, 65536)
