@@ -251,6 +251,8 @@ def main():
                     help="softmax + cross-entropy on labels (the benchmark's workload) or the paper's tanh outputs with "
                          "summed squared error on a dense target matrix")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--exchange", default="allreduce", choices=["allreduce", "ordered"],
+                    help="gradient exchange over several GPUs: NCCL all-reduce, or all-gather + sum in rank order")
     ap.add_argument("--patterns", type=int, default=0,
                     help="patterns per GPU instead of the workload's own count (for profiler captures of a smaller case)")
     args = ap.parse_args()
@@ -302,7 +304,7 @@ def main():
     net = ul.Mlp(sizes, math_mode, chunk)
     lr = 1e-3 / (batch * world)
     stream = torch.cuda.current_stream()
-    exchange = dp.GradientExchange(dW + db, dist)
+    exchange = dp.GradientExchange(dW + db, dist, ordered=args.exchange == "ordered")
 
     def step(Xd, yd, host=None):
         for i, lo in enumerate(starts):
@@ -462,7 +464,7 @@ def main():
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if args.math == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": "%s: %s MLP, %d patterns per GPU, seed %d" % (args.workload, "-".join(map(str, sizes)), batch, seed),
-                   "math": args.math, "head": args.head, "global_batch": batch * world, "parallelism": "dp%d" % world,
+                   "math": args.math, "head": args.head, "global_batch": batch * world, "parallelism": "dp%d" % world, "exchange": args.exchange if world > 1 else None,
                    "l2": "no flush: inputs and intermediates of a step (X %.0f MB, logits %.0f MB) exceed the 126 MB L2"
                          % (batch * sizes[0] * 4 / 1e6, batch * sizes[-1] * 4 / 1e6),
                    "step": "gradient evaluation + W -= lr*grad, lr = 1e-3 / global_batch"},

@@ -26,14 +26,21 @@ def split_range(n_patterns: int, world: int, rank: int):
 
 
 class GradientExchange:
-    """Sums per-rank gradients in place.  One flat buffer is kept, so an exchange is one all-reduce for all
-    gradient tensors plus one for the loss."""
+    """Sums per-rank gradients in place.  One flat buffer is kept, so an exchange is one collective for all
+    gradient tensors plus one for the loss.
 
-    def __init__(self, tensors, dist=None):
+    ordered=False: all-reduce (the library picks the order of the additions).
+    ordered=True:  all-gather, then every rank adds the per-rank vectors in rank order: the sum does not depend on
+                   the collective's algorithm and is bitwise the same on every rank (the on-device reductions of the
+                   library are fixed-order too, so the whole evaluation then repeats bit for bit)."""
+
+    def __init__(self, tensors, dist=None, ordered=False):
         import torch
         self.dist = dist
+        self.ordered = ordered
         self.sizes = [int(t.numel()) for t in tensors]
         self.flat = torch.empty(sum(self.sizes), dtype=tensors[0].dtype, device=tensors[0].device)
+        self.gathered = None
 
     def all_reduce(self, tensors, loss):
         """tensors: list of gradient tensors (same shapes as at construction); loss: 1-element tensor."""
@@ -41,9 +48,28 @@ class GradientExchange:
         if self.dist is None or self.dist.get_world_size() == 1:
             return
         torch.cat([t.reshape(-1) for t in tensors], out=self.flat)
-        self.dist.all_reduce(self.flat)
+        if self.ordered:
+            world = self.dist.get_world_size()
+            n = self.flat.numel()
+            if self.gathered is None:
+                # one row per rank; the loss has its own dtype (double) and travels in its own gather below
+                self.gathered = torch.empty(world * n, dtype=self.flat.dtype, device=self.flat.device)
+            self.dist.all_gather_into_tensor(self.gathered, self.flat)
+            parts = self.gathered.view(world, n)
+            self.flat.copy_(parts[0])
+            for r in range(1, world):
+                self.flat.add_(parts[r])
+            losses = torch.empty(world * loss.numel(), dtype=loss.dtype, device=loss.device)
+            self.dist.all_gather_into_tensor(losses, loss.reshape(-1))
+            lp = losses.view(world, -1)
+            acc = lp[0].clone()
+            for r in range(1, world):
+                acc.add_(lp[r])
+            loss.copy_(acc.view_as(loss))
+        else:
+            self.dist.all_reduce(self.flat)
+            self.dist.all_reduce(loss)
         off = 0
         for t, n in zip(tensors, self.sizes):
             t.copy_(self.flat[off:off + n].view_as(t))
             off += n
-        self.dist.all_reduce(loss)

@@ -25,7 +25,7 @@ def _free_port():
         return s.getsockname()[1]
 
 
-def _worker(rank, world, port, out_dir):
+def _worker(rank, world, port, out_dir, ordered=False):
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
@@ -36,7 +36,7 @@ def _worker(rank, world, port, out_dir):
         loss, dW, db = oracle.mlp_gradient(Ws, bs, X, y)
         grads = [torch.from_numpy(np.ascontiguousarray(g)) for g in dW + db]       # float64 on the CPU
         loss_t = torch.tensor([loss], dtype=torch.float64)
-        ex = dp.GradientExchange(grads, dist)
+        ex = dp.GradientExchange(grads, dist, ordered=ordered)
         ex.all_reduce(grads, loss_t)
         np.savez(os.path.join(out_dir, "rank%d.npz" % rank), loss=loss_t.numpy(), *[g.numpy() for g in grads])
     finally:
@@ -54,6 +54,24 @@ def test_two_ranks_sum_to_the_full_batch(tmp_path):
         assert abs(got["loss"][0] - loss) <= 1e-12 * abs(loss)
         for i, ref in enumerate(dW + db):
             assert np.allclose(got["arr_%d" % i], ref, rtol=1e-12, atol=1e-14)
+
+
+def test_ordered_exchange_is_the_rank_order_sum_on_every_rank(tmp_path):
+    world = 2
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path), True), nprocs=world, join=True)
+    Ws, bs = si.mlp_params(SEED, SIZES)
+    per_rank = []
+    for rank in range(world):
+        first, last = dp.shard_range(rank, world, PER_RANK)
+        X, y = si.mlp_batch(SEED, SIZES, last - first, offset=first)
+        per_rank.append(oracle.mlp_gradient(Ws, bs, X, y))
+    got = [np.load(os.path.join(str(tmp_path), "rank%d.npz" % rank)) for rank in range(world)]
+    assert got[0]["loss"][0] == got[1]["loss"][0] == per_rank[0][0] + per_rank[1][0]
+    n_tensors = 2 * (len(SIZES) - 1)
+    for i in range(n_tensors):
+        a0 = (per_rank[0][1] + per_rank[0][2])[i]; a1 = (per_rank[1][1] + per_rank[1][2])[i]
+        assert np.array_equal(got[0]["arr_%d" % i], got[1]["arr_%d" % i])       # bitwise the same on both ranks
+        assert np.array_equal(got[0]["arr_%d" % i], a0 + a1)                     # and exactly rank 0's plus rank 1's
 
 
 def test_shard_arithmetic():
