@@ -41,14 +41,14 @@ NOMINAL_TF32_OVER_BF16 = 0.5        # dense TF32 tensor rate is half the BF16 ra
 # the pattern count (profiles/tc_gemm_3xtf32_config3.md, profiles/bf16_gemm_config3.md).  Only reported while the
 # library still is the version the counters were taken on.
 NCU_TRAFFIC = {
-    "library_version": 104,
+    "library_version": 105,
     # dram__bytes_read.sum + dram__bytes_write.sum per launch, captured at 16384 patterns (x4) / 32768 patterns (x2)
-    ("config3", "3xtf32", (3203, 481, 65536)): 4 * (301.950464e6 + 19.559936e6),
-    ("config3", "3xtf32", (65536, 480, 3203)): 4 * (309.913600e6 + 19.342336e6),
-    ("config3", "3xtf32", (65536, 3203, 480)): 4 * (77.489664e6 + 163.489280e6),
-    ("config3", "bf16", (65536, 3203, 480)): 2 * (38.357248e6 + 171.255040e6),
-    ("config3", "bf16", (3203, 481, 65536)): 2 * (253.020416e6 + 18.108416e6),
-    ("config3", "bf16", (65536, 480, 3203)): 2 * (251.651328e6 + 18.018048e6),
+    ("config3", "3xtf32", (3203, 481, 65536)): 4 * (302.09715e6 + 24.203776e6),
+    ("config3", "3xtf32", (65536, 480, 3203)): 4 * (309.96019e6 + 25.910528e6),
+    ("config3", "3xtf32", (65536, 3203, 480)): 4 * (77.244928e6 + 168.68992e6),
+    ("config3", "bf16", (65536, 3203, 480)): 2 * (38.540544e6 + 172.197632e6),
+    ("config3", "bf16", (3203, 481, 65536)): 2 * (253.675520e6 + 17.889792e6),
+    ("config3", "bf16", (65536, 480, 3203)): 2 * (250.972416e6 + 18.076160e6),
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
