@@ -3,8 +3,8 @@
  * single-precision matrix products, on one NVIDIA B200 (sm_100a).
  *
  * The calls follow the problem statement of "Ultra-Large-Scale Neural-Network
- * Training on a PIII Cluster": a Level-3-BLAS SGEMM (Section 3.1), "compute the
- * error" and "compute the gradient" of a block of training patterns (Sections
+ * Training on a PIII Cluster": a Level-3-BLAS SGEMM (Section 3.1), the error and
+ * the gradient of a block of training patterns (Sections
  * 4.2-4.3, 6.2) and the plain step W := W - alpha*grad (Section 4.2).
  *
  * Conventions that hold for every call
