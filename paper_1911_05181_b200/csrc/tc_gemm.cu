@@ -81,7 +81,7 @@ struct TcParams {
     int chunk_blocks;       // k-blocks accumulated on one TMEM accumulator before it is added into the tile total
     int fast_math;          // TF32 mode: approximate exp
     int c_tma;              // the output (C or the split-K partials) is written with TMA stores
-    int producers;          // producer warps that have something to fetch (2 or 3)
+    int producers;          // producer warps that have something to fetch (1, 2 or 3)
     int direct;             // CTA pairs without an operand pass: both CTAs count their landed bytes on CTA 0's `full`
                             // barriers (cta_group::2 loads), nothing is relayed
     int64_t n_patterns, n_classes;      // bounds of the logits operand when a_transform
@@ -197,8 +197,11 @@ __device__ __forceinline__ void split4(const float4 x, float4& hi, float4& lo) {
     lo = make_float4(to_tf32(x.x - hi.x), to_tf32(x.y - hi.y), to_tf32(x.z - hi.z), to_tf32(x.w - hi.w));
 }
 
-template <int EPI, int CG>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// MULTI: the product has no operand pass; its copies are then issued by three warps and, in a CTA pair, counted on CTA 0's
+// barriers.  Products with an operand pass are compiled without any of that (and launched without the two extra warps):
+// they ran 1-4 % slower with it in the same kernel.
+template <int EPI, int CG, bool MULTI>
+__global__ void __launch_bounds__(MULTI ? NUM_THREADS : FIRST_EXTRA_PRODUCER * 32, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_a_lo, const __grid_constant__ CUtensorMap map_b_lo,
                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c_lo, const TcParams p) {
@@ -211,6 +214,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const GemmDesc& d = p.d;
+    constexpr bool SPLIT = !MULTI;              // an operand pass runs (warps 6-13)
+    constexpr bool DIRECT = MULTI && CG == 2;   // both CTAs of a pair count their landed bytes on CTA 0's `full` barriers
     // With CG == 2 the two CTAs of a cluster work on the same sequence of tiles.  CTA 0 issues the products.  Its
     // `ready` barriers collect its own operand-pass warps and, per stage, 8 transaction bytes that warp 1 of CTA 1
     // sends over with an asynchronous store when CTA 1's stage is ready (an arrival on another CTA's barrier holds
@@ -221,9 +226,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&ctrl->full[s]), p.producers);      // one arrival (with its byte count) per producer warp at work
+            mbar_init(smem_u32(&ctrl->full[s]), MULTI ? p.producers : 1);      // one arrival (with its byte count) per producer warp at work
             // CTA 0: its own operand-pass warps plus one arrival relayed from CTA 1; CTA 1: its operand-pass warps
-            const int ready_count = (p.split_pass ? NUM_SPLIT_WARPS : 0) + ((CG == 2 && rank == 0 && !p.direct) ? 1 : 0);
+            const int ready_count = (SPLIT ? NUM_SPLIT_WARPS : 0) + ((CG == 2 && rank == 0 && !DIRECT) ? 1 : 0);
             mbar_init(smem_u32(&ctrl->ready[s]), ready_count > 0 ? ready_count : 1);      // unused when nothing arrives on it
             mbar_init(smem_u32(&ctrl->empty[s]), 1);
         }
@@ -249,7 +254,71 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int off_a_hi = 0, off_b_hi = A_TILE_BYTES;
     const int off_a_lo = A_TILE_BYTES + p.b_tile_bytes, off_b_lo = 2 * A_TILE_BYTES + p.b_tile_bytes;
 
-    if (warp == 0 || warp >= FIRST_EXTRA_PRODUCER) {
+    if (!MULTI && warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (products with an operand pass:
+        // one warp fetches everything; the extra polling warps cost such products 3-5 %)
+        RingPos rp{0, 0};
+        bool ok = true;
+        for (int u = first_unit; u < p.units && ok; u += unit_step) {
+            int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
+            int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+            // this CTA's rows of A and its share of the tile's columns of B
+            const int b_cols = tile_cols(p, nt) / CG;
+            const int m0 = (mt * CG + rank) * BM, n0 = nt * p.bn + rank * b_cols;
+            // a K-major B tile is one box of bn/CG rows (rows past the matrix arrive as zeros); an MN-major one is
+            // a box per 32 columns, and only the boxes the products read are fetched
+            const int b_boxes = b_cols >> 5;
+            const uint32_t b_bytes = (uint32_t)(p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes);
+            const uint32_t tx_bytes = (uint32_t)A_TILE_BYTES * (p.a_pre ? 2u : 1u) + b_bytes * (p.b_pre ? 2u : 1u);
+            int k0 = (int)kbeg;
+            for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
+                const int s = rp.stage;
+                if (!wait_bar_warp(&ctrl->empty[s], rp.phase ^ 1, ctrl, p.status)) { ok = false; break; }
+                rp.advance(p.stages);
+                const uint32_t bar = smem_u32(&ctrl->full[s]);
+                const uint32_t sa = smem_u32(stage_base + (size_t)s * p.stage_bytes + off_a_hi);
+                const uint32_t sb = sa + off_b_hi;
+                if (elect_one()) {
+                    mbar_expect_tx(bar, tx_bytes);
+                    if (!p.a_mn) {
+                        tma_load_2d(sa, &map_a, k0, m0, bar);                       // box {BK k, 128 rows}
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < BM / 32; ++g)                           // boxes {32 m, BK k}
+                            tma_load_2d(sa + g * (BK * 128), &map_a, m0 + 32 * g, k0, bar);
+                    }
+                    if (!p.b_mn) {
+                        tma_load_2d(sb, &map_b, k0, n0, bar);                       // box {BK k, bn/CG rows}
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < BN_MAX / 32; ++g)
+                            if (g < b_boxes) tma_load_2d(sb + g * (BK * 128), &map_b, n0 + 32 * g, k0, bar);
+                    }
+                    // operands stored as (hi, lo) pairs: the lo tiles land beside the hi tiles
+                    if (p.a_pre) {
+                        const uint32_t sal = sa + off_a_lo;
+                        if (!p.a_mn) {
+                            tma_load_2d(sal, &map_a_lo, k0, m0, bar);
+                        } else {
+#pragma unroll
+                            for (int g = 0; g < BM / 32; ++g) tma_load_2d(sal + g * (BK * 128), &map_a_lo, m0 + 32 * g, k0, bar);
+                        }
+                    }
+                    if (p.b_pre) {
+                        const uint32_t sbl = sa + off_b_lo;
+                        if (!p.b_mn) {
+                            tma_load_2d(sbl, &map_b_lo, k0, n0, bar);
+                        } else {
+#pragma unroll
+                            for (int g = 0; g < BN_MAX / 32; ++g)
+                                if (g < b_boxes) tma_load_2d(sbl + g * (BK * 128), &map_b_lo, n0 + 32 * g, k0, bar);
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    } else if (MULTI && (warp == 0 || warp >= FIRST_EXTRA_PRODUCER)) {
         // ------------------------------------------------------------------ TMA producers
         // role 0: the A tiles (and their lo halves when both operands are stored pairs); role 1: the B tiles;
         // role 2: the lo halves of B, or those of A when only A is a stored pair
@@ -270,18 +339,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t b_bytes = (uint32_t)(p.b_mn ? b_boxes * (BK * 128) : p.b_tile_bytes);
             // what this warp fetches per stage; with direct counting CTA 0 announces the bytes of both CTAs
             const uint32_t tx_bytes = ((get_a ? (uint32_t)A_TILE_BYTES : 0u) + (get_a_lo ? (uint32_t)A_TILE_BYTES : 0u) +
-                                       (get_b ? b_bytes : 0u) + (get_b_lo ? b_bytes : 0u)) * (p.direct ? (uint32_t)CG : 1u);
+                                       (get_b ? b_bytes : 0u) + (get_b_lo ? b_bytes : 0u)) * (DIRECT ? (uint32_t)CG : 1u);
             int k0 = (int)kbeg;
             for (int kb = 0; kb < nkb; ++kb, k0 += BK) {
                 const int s = rp.stage;
                 if (!wait_bar_warp(&ctrl->empty[s], rp.phase ^ 1, ctrl, p.status)) { ok = false; break; }
                 rp.advance(p.stages);
                 const uint32_t bar_local = smem_u32(&ctrl->full[s]);
-                const uint32_t bar = (CG == 2 && p.direct) ? addr_in_rank0(bar_local) : bar_local;
+                const uint32_t bar = (CG == 2 && DIRECT) ? addr_in_rank0(bar_local) : bar_local;
                 const uint32_t sa = smem_u32(stage_base + (size_t)s * p.stage_bytes + off_a_hi);
                 const uint32_t sb = sa + off_b_hi;
                 auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
-                    if (CG == 2 && p.direct) tma_load_2d_pair(dst, map, x, y, bar); else tma_load_2d(dst, map, x, y, bar);
+                    if (CG == 2 && DIRECT) tma_load_2d_pair(dst, map, x, y, bar); else tma_load_2d(dst, map, x, y, bar);
                 };
                 auto load_a = [&](uint32_t dst, const CUtensorMap* map) {
                     if (!p.a_mn) {
@@ -301,7 +370,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                 };
                 if (elect_one()) {
-                    if (!p.direct || rank == 0) mbar_expect_tx(bar_local, tx_bytes);
+                    if (!DIRECT || rank == 0) mbar_expect_tx(bar_local, tx_bytes);
                     if (get_a) load_a(sa, &map_a);
                     if (get_b) load_b(sb, &map_b);
                     // operands stored as (hi, lo) pairs: the lo tiles land beside the hi tiles
@@ -356,12 +425,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         d_tmem = tmem_base + reg * BN_MAX;
                     }
                     const int s = rp.stage;
-                    if (!p.split_pass && !wait_bar_warp(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
+                    if (!SPLIT && !wait_bar_warp(&ctrl->full[s], rp.phase, ctrl, p.status)) { ok = false; break; }
                     // CTA 1's signal for this stage completes 8 transaction bytes on `ready`; posting the expectation is
                     // this warp's own arrival on it (not needed when CTA 1's bytes are counted on `full` directly)
-                    const bool relayed = CG == 2 && !p.direct;
+                    const bool relayed = CG == 2 && !DIRECT;
                     if (relayed && elect_one()) mbar_expect_tx(smem_u32(&ctrl->ready[s]), 8);
-                    if ((p.split_pass || relayed) && !wait_bar_warp(&ctrl->ready[s], rp.phase, ctrl, p.status)) { ok = false; break; }
+                    if ((SPLIT || relayed) && !wait_bar_warp(&ctrl->ready[s], rp.phase, ctrl, p.status)) { ok = false; break; }
                     rp.advance(p.stages);
                     tc_fence_after();
                     const uint32_t soff = (uint32_t)s * stage_inc;
@@ -391,7 +460,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
             }
         }
-        if (CG == 2 && rank == 1 && !p.direct) {
+        if (CG == 2 && rank == 1 && !DIRECT) {
             // CTA 1 issues nothing: this warp tells CTA 0 when a stage of CTA 1 is ready for the products
             RingPos rp{0, 0};
             bool ok = true;
@@ -400,7 +469,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
                 for (int kb = 0; kb < nkb; ++kb) {
                     const int s = rp.stage;
-                    uint64_t* bar = p.split_pass ? &ctrl->ready[s] : &ctrl->full[s];
+                    uint64_t* bar = SPLIT ? &ctrl->ready[s] : &ctrl->full[s];
                     if (!wait_bar_warp(bar, rp.phase, ctrl, p.status)) { ok = false; break; }
                     rp.advance(p.stages);
                     if (lane == 0) signal_rank0(smem_u32(&ctrl->relay_sink[s]), smem_u32(&ctrl->ready[s]));
@@ -664,7 +733,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
         if (lane == 0) bulk_wait_all();         // every store of this warp has left shared memory and is complete
-    } else if (p.split_pass) {
+    } else if (SPLIT) {
         // ------------------------------------------------------------------ operand pass (lo parts, logits -> delta)
         const int st = threadIdx.x - (2 + NUM_EPI_WARPS) * 32;          // 0..255
         constexpr int NT = NUM_SPLIT_WARPS * 32;
@@ -880,17 +949,17 @@ int* status_ptr() {
 
 struct Maps { CUtensorMap a, b, a_lo, b_lo, c, c_lo; };
 
-template <int EPI, int CG>
+template <int EPI, int CG, bool MULTI>
 ulsnn_status_t launch(const Maps& m, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<EPI, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
+        if (cudaFuncSetAttribute(tc_gemm_kernel<EPI, CG, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
             return ULSNN_ERR_CUDA;
         configured = true;
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
-    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.blockDim = dim3(MULTI ? NUM_THREADS : FIRST_EXTRA_PRODUCER * 32, 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -898,14 +967,16 @@ ulsnn_status_t launch(const Maps& m, const TcParams& p, int smem_bytes, int grid
     attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG>, m.a, m.b, m.a_lo, m.b_lo, m.c, m.c_lo, p);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG, MULTI>, m.a, m.b, m.a_lo, m.b_lo, m.c, m.c_lo, p);
     count_launch(1);
     return cuda_ok(e == cudaSuccess ? cudaGetLastError() : e);
 }
 
 template <int EPI>
 ulsnn_status_t launch_cg(int cg, const Maps& m, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
-    return cg == 2 ? launch<EPI, 2>(m, p, smem_bytes, grid, stream) : launch<EPI, 1>(m, p, smem_bytes, grid, stream);
+    if (p.split_pass)
+        return cg == 2 ? launch<EPI, 2, false>(m, p, smem_bytes, grid, stream) : launch<EPI, 1, false>(m, p, smem_bytes, grid, stream);
+    return cg == 2 ? launch<EPI, 2, true>(m, p, smem_bytes, grid, stream) : launch<EPI, 1, true>(m, p, smem_bytes, grid, stream);
 }
 
 }  // namespace
@@ -963,7 +1034,7 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     p.a_pre = (three_x && d.A_lo && !d.a_transform) ? 1 : 0;
     p.b_pre = (three_x && d.B_lo) ? 1 : 0;
     p.split_pass = (d.a_transform || (three_x && !(p.a_pre && p.b_pre))) ? 1 : 0;
-    p.producers = 2 + ((p.a_pre || p.b_pre) ? 1 : 0);
+    p.producers = p.split_pass ? 1 : 2 + ((p.a_pre || p.b_pre) ? 1 : 0);
     p.direct = (cg == 2 && !p.split_pass) ? 1 : 0;
     p.fast_math = three_x ? 0 : 1;
     p.chunk_blocks = three_x ? 256 / BK : (1 << 30);       // 256 elements of K per accumulator in the accurate mode
