@@ -200,7 +200,8 @@ __device__ __forceinline__ void split4(const float4 x, float4& hi, float4& lo) {
 // MULTI: the product has no operand pass; its copies are then issued by three warps and, in a CTA pair, counted on CTA 0's
 // barriers.  Products with an operand pass are compiled without any of that (and launched without the two extra warps):
 // they ran 1-4 % slower with it in the same kernel.
-template <int EPI, int CG, bool MULTI>
+// THREE_X: the 3xTF32 mode (three products per k step on (hi, lo) pairs, accurate exp) against plain TF32.
+template <int EPI, int CG, bool MULTI, bool THREE_X>
 __global__ void __launch_bounds__(MULTI ? NUM_THREADS : FIRST_EXTRA_PRODUCER * 32, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_a_lo, const __grid_constant__ CUtensorMap map_b_lo,
@@ -441,7 +442,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const uint64_t a_hi = da_hi0 + (uint64_t)(soff + ks * a_kinc);
                         const uint64_t b_hi = db_hi0 + (uint64_t)(soff + ks * b_kinc);
                         const uint32_t accumulate = (chunk_start && ks == 0) ? 0u : 1u;
-                        if (p.three_x) {
+                        if (THREE_X) {
                             const uint64_t a_lo = da_lo0 + (uint64_t)(soff + ks * a_kinc);
                             const uint64_t b_lo = db_lo0 + (uint64_t)(soff + ks * b_kinc);
                             umma_tf32<CG>(d_tmem, a_lo, b_hi, idesc, accumulate);
@@ -629,7 +630,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             }
                             run_s = (run_m == -INFINITY ? 0.f : run_s * exp_t<FAST>(run_m - nm)) + s;
                         };
-                        if (p.fast_math) sum_exp(std::true_type{}); else sum_exp(std::false_type{});
+                        sum_exp(std::integral_constant<bool, !THREE_X>{});
                         run_m = nm;
 #pragma unroll
                         for (int q8 = 0; q8 < BN_MAX / 32; ++q8) if (q8 == c) tile_max[q8] = nm;      // static indices: stays in registers
@@ -855,7 +856,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                     }
                 };
-                if (p.three_x) pass(std::true_type{}); else pass(std::false_type{});
+                pass(std::integral_constant<bool, THREE_X>{});
                 proxy_fence_async();            // make these generic-proxy writes visible to the tensor core's reads
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->ready[s]));
@@ -949,11 +950,11 @@ int* status_ptr() {
 
 struct Maps { CUtensorMap a, b, a_lo, b_lo, c, c_lo; };
 
-template <int EPI, int CG, bool MULTI>
+template <int EPI, int CG, bool MULTI, bool THREE_X>
 ulsnn_status_t launch(const Maps& m, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<EPI, CG, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
+        if (cudaFuncSetAttribute(tc_gemm_kernel<EPI, CG, MULTI, THREE_X>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
             return ULSNN_ERR_CUDA;
         configured = true;
     }
@@ -967,16 +968,21 @@ ulsnn_status_t launch(const Maps& m, const TcParams& p, int smem_bytes, int grid
     attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG, MULTI>, m.a, m.b, m.a_lo, m.b_lo, m.c, m.c_lo, p);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG, MULTI, THREE_X>, m.a, m.b, m.a_lo, m.b_lo, m.c, m.c_lo, p);
     count_launch(1);
     return cuda_ok(e == cudaSuccess ? cudaGetLastError() : e);
+}
+
+template <int EPI, bool MULTI, bool THREE_X>
+ulsnn_status_t launch_cg2(int cg, const Maps& m, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
+    return cg == 2 ? launch<EPI, 2, MULTI, THREE_X>(m, p, smem_bytes, grid, stream) : launch<EPI, 1, MULTI, THREE_X>(m, p, smem_bytes, grid, stream);
 }
 
 template <int EPI>
 ulsnn_status_t launch_cg(int cg, const Maps& m, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
     if (p.split_pass)
-        return cg == 2 ? launch<EPI, 2, false>(m, p, smem_bytes, grid, stream) : launch<EPI, 1, false>(m, p, smem_bytes, grid, stream);
-    return cg == 2 ? launch<EPI, 2, true>(m, p, smem_bytes, grid, stream) : launch<EPI, 1, true>(m, p, smem_bytes, grid, stream);
+        return p.three_x ? launch_cg2<EPI, false, true>(cg, m, p, smem_bytes, grid, stream) : launch_cg2<EPI, false, false>(cg, m, p, smem_bytes, grid, stream);
+    return p.three_x ? launch_cg2<EPI, true, true>(cg, m, p, smem_bytes, grid, stream) : launch_cg2<EPI, true, false>(cg, m, p, smem_bytes, grid, stream);
 }
 
 }  // namespace
