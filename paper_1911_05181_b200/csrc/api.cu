@@ -220,7 +220,7 @@ extern "C" const char* ulsnn_status_string(ulsnn_status_t s) {
     return "unknown status";
 }
 
-extern "C" int ulsnn_version(void) { return 107; }
+extern "C" int ulsnn_version(void) { return 108; }
 
 extern "C" void ulsnn_launch_counts(int64_t counts[4]) {
     for (int i = 0; i < 4; ++i) counts[i] = g_counts[i].load(std::memory_order_relaxed);

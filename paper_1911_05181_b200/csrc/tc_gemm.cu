@@ -2,15 +2,16 @@
 // the error-compensated 3xTF32 mode (operands as TF32 hi/lo pairs, split on chip or loaded as stored pairs),
 // and the fused epilogues.
 //
-// One persistent CTA per SM, 16 warps with fixed roles:
-//   warps 0,14,15 TMA producers   global -> swizzled shared-memory stages (cp.async.bulk.tensor, no multicast):
-//                                 warp 0 the A tiles, warp 14 the B tiles, warp 15 the lo halves of stored pairs
+// One persistent CTA per SM, warps with fixed roles (14 warps in the variants with an operand pass, 8 in those without):
+//   warp 0 (+ 6, 7) TMA producers global -> swizzled shared-memory stages (cp.async.bulk.tensor, no multicast); in the
+//                                 variants without an operand pass warp 0 fetches the A tiles, warp 6 the B tiles and
+//                                 warp 7 the lo halves of stored pairs
 //   warp 1      product issuer    all lanes run the loop, an elected lane issues tcgen05.mma.kind::tf32 and the
 //                                 commits (in the second CTA of a pair: relays "stage ready" to the first)
 //   warps 2-5   epilogue          tcgen05.ld of the 128 x BN fp32 accumulator (one row per thread), fused math, then
 //                                 32x32 blocks staged in swizzled shared memory and written with TMA stores
 //                                 (whole 128-byte lines, edges clipped by the tensor map)
-//   warps 6-13  operand pass      for operands that do not arrive as stored pairs (3xTF32), or when A is formed
+//   warps 6-13  operand pass      (variants with a pass) for operands that do not arrive as stored pairs (3xTF32), or when A is formed
 //                                 from logits: reads a landed stage, rewrites it as hi = tf32_rn(x) and writes
 //                                 lo = tf32_rn(x - hi) beside it
 // Tiles: 128 x BN (BN <= 256) by one CTA, or 256 x BN by the two CTAs of a cluster (tcgen05 cta_group::2): each
@@ -54,9 +55,10 @@ constexpr int NUM_SPLIT_WARPS = 8;
 constexpr int NUM_PRODUCERS = 3;         // warp 0 and the last two warps: a thread gets its next TMA copy accepted only
                                         // some hundred nanoseconds after the previous one, so the copies of a stage
                                         // are spread over three issuing threads
-constexpr int FIRST_EXTRA_PRODUCER = 2 + NUM_EPI_WARPS + NUM_SPLIT_WARPS;
-constexpr int NUM_WARPS = FIRST_EXTRA_PRODUCER + NUM_PRODUCERS - 1;
-constexpr int NUM_THREADS = NUM_WARPS * 32;
+// Variants with an operand pass: warps 0 (producer), 1 (issuer), 2-5 (epilogue), 6-13 (operand pass): 448 threads.
+// Variants without: warps 0, 1, 2-5 and the two extra producers 6-7: 256 threads, so the epilogue may use more registers.
+constexpr int first_extra_producer(bool multi) { return 2 + NUM_EPI_WARPS + (multi ? 0 : NUM_SPLIT_WARPS); }
+constexpr int threads_of(bool multi) { return (first_extra_producer(multi) + (multi ? NUM_PRODUCERS - 1 : 0)) * 32; }
 constexpr int MAX_STAGES = 12;
 constexpr int NUM_SMS = 148;               // B200; fixes the tile schedule (and with it every summation order)
 constexpr int A_TILE_BYTES = BM * BK * 4;
@@ -202,7 +204,7 @@ __device__ __forceinline__ void split4(const float4 x, float4& hi, float4& lo) {
 // they ran 1-4 % slower with it in the same kernel.
 // THREE_X: the 3xTF32 mode (three products per k step on (hi, lo) pairs, accurate exp) against plain TF32.
 template <int EPI, int CG, bool MULTI, bool THREE_X>
-__global__ void __launch_bounds__(MULTI ? NUM_THREADS : FIRST_EXTRA_PRODUCER * 32, 1)
+__global__ void __launch_bounds__(threads_of(MULTI), 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_a_lo, const __grid_constant__ CUtensorMap map_b_lo,
                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c_lo, const TcParams p) {
@@ -215,6 +217,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const GemmDesc& d = p.d;
+    constexpr int FIRST_EXTRA = 2 + NUM_EPI_WARPS + (MULTI ? 0 : NUM_SPLIT_WARPS);      // first of the two extra producer warps
     constexpr bool SPLIT = !MULTI;              // an operand pass runs (warps 6-13)
     constexpr bool DIRECT = MULTI && CG == 2;   // both CTAs of a pair count their landed bytes on CTA 0's `full` barriers
     // With CG == 2 the two CTAs of a cluster work on the same sequence of tiles.  CTA 0 issues the products.  Its
@@ -319,11 +322,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 __syncwarp();
             }
         }
-    } else if (MULTI && (warp == 0 || warp >= FIRST_EXTRA_PRODUCER)) {
+    } else if (MULTI && (warp == 0 || warp >= FIRST_EXTRA)) {
         // ------------------------------------------------------------------ TMA producers
         // role 0: the A tiles (and their lo halves when both operands are stored pairs); role 1: the B tiles;
         // role 2: the lo halves of B, or those of A when only A is a stored pair
-        const int role = warp == 0 ? 0 : warp - FIRST_EXTRA_PRODUCER + 1;
+        const int role = warp == 0 ? 0 : warp - FIRST_EXTRA + 1;
         const bool get_a = role == 0, get_b = role == 1;
         const bool get_a_lo = p.a_pre && (p.b_pre ? role == 0 : role == 2), get_b_lo = p.b_pre && role == 2;
         RingPos rp{0, 0};
@@ -960,7 +963,7 @@ ulsnn_status_t launch(const Maps& m, const TcParams& p, int smem_bytes, int grid
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
-    cfg.blockDim = dim3(MULTI ? NUM_THREADS : FIRST_EXTRA_PRODUCER * 32, 1, 1);
+    cfg.blockDim = dim3(threads_of(MULTI), 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
