@@ -239,6 +239,53 @@ def run_sgemm_sweep(args):
     return 0
 
 
+def run_peaks(args):
+    """--workload peaks: the denominators measured directly on this GPU with library routines (never on the library's
+    own path): torch.matmul 8192^3 with TF32 allowed and in bf16, each as the best of 10 isolated calls (burst) and
+    back to back for 4 s (sustained, under the power cap), with the SM clock sampled during the sustained loop."""
+    import torch
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return 0
+    n = 8192
+    out = {"workload": "peaks", "n": n, "nominal_tf32_tflops": 1100.0, "nominal_bf16_tflops": 2250.0}
+    for name, dtype, tf32 in (("tf32", torch.float32, True), ("bf16", torch.bfloat16, False)):
+        torch.backends.cuda.matmul.allow_tf32 = tf32
+        a = torch.randn(n, n, device="cuda", dtype=dtype); b = torch.randn(n, n, device="cuda", dtype=dtype)
+        c = torch.empty(n, n, device="cuda", dtype=dtype)
+        for _ in range(3):
+            torch.matmul(a, b, out=c)
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(10):
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(); torch.matmul(a, b, out=c); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+            time.sleep(0.05)
+        sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+        sampler.start()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        reps = 0
+        t0 = time.perf_counter()
+        e0.record()
+        while time.perf_counter() - t0 < 4.0:
+            for _ in range(20):
+                torch.matmul(a, b, out=c)
+            reps += 20
+            torch.cuda.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        out[name] = {"burst_tflops": 2.0 * n ** 3 / (best * 1e-3) / 1e12,
+                     "sustained_tflops": 2.0 * n ** 3 * reps / (e0.elapsed_time(e1) * 1e-3) / 1e12,
+                     "sustained_clocks": clocks}
+        time.sleep(1.0)
+    torch.backends.cuda.matmul.allow_tf32 = False
+    print(json.dumps(out))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -246,7 +293,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--math", default="3xtf32", choices=sorted(MATH))
-    ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS) + ["sgemm"])
+    ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS) + ["sgemm", "peaks"])
     ap.add_argument("--head", default="softmax", choices=["softmax", "sse"],
                     help="softmax + cross-entropy on labels (the benchmark's workload) or the paper's tanh outputs with "
                          "summed squared error on a dense target matrix")
@@ -256,6 +303,8 @@ def main():
     ap.add_argument("--patterns", type=int, default=0,
                     help="patterns per GPU instead of the workload's own count (for profiler captures of a smaller case)")
     args = ap.parse_args()
+    if args.workload == "peaks":
+        return run_peaks(args) if args.impl == "ours" else 0
     if args.workload == "sgemm":
         return run_sgemm_sweep(args) if args.impl == "ours" else 0
     if args.impl == "reference":

@@ -163,6 +163,42 @@ def mlp_probe(Ws, bs, X, want_probs=True, want_hidden=True):
     return probs, hid
 
 
+def sgemm_abs(transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C=None, ldc=0) -> np.ndarray:
+    """|alpha| * |op(A)| * |op(B)| + |beta| * |C|: the magnitude sums the forward error of the product is proportional to."""
+    A = _f32(A); B = _f32(B)
+    out = np.empty((M, N), dtype=np.float64)
+    if beta != 0.0:
+        C = _f32(C)
+    _load().oracle_sgemm_abs(
+        ctypes.c_int(_trans(transA)), ctypes.c_int(_trans(transB)),
+        ctypes.c_int64(M), ctypes.c_int64(N), ctypes.c_int64(K), ctypes.c_double(alpha),
+        _ptr(A, ctypes.c_float), ctypes.c_int64(lda), _ptr(B, ctypes.c_float), ctypes.c_int64(ldb),
+        ctypes.c_double(beta), _ptr(C if beta != 0.0 else None, ctypes.c_float), ctypes.c_int64(ldc),
+        _ptr(out, ctypes.c_double))
+    return out
+
+
+def mlp_gradient_abs(Ws, bs, X, labels=None, T=None):
+    """([aW_l], [ab_l]): the summed gradient's back-propagation with every term in absolute value (softmax head when
+    `labels` is given, the paper's tanh + squared-error head when `T` is).  What rounding errors are proportional to."""
+    sizes, Wflat, bflat = _flatten(Ws, bs)
+    X = np.ascontiguousarray(_f32(X))
+    head = 0 if T is None else 1
+    if head == 0:
+        labels = np.ascontiguousarray(labels, dtype=np.int32)
+    else:
+        T = np.ascontiguousarray(_f32(T))
+    aW = np.zeros(Wflat.size, dtype=np.float64); ab = np.zeros(bflat.size, dtype=np.float64)
+    rc = _load().oracle_mlp_gradient_abs(
+        ctypes.c_int(len(Ws)), _ptr(sizes, ctypes.c_int32), _ptr(Wflat, ctypes.c_float),
+        _ptr(bflat, ctypes.c_float), _ptr(X, ctypes.c_float), ctypes.c_int64(X.shape[1]),
+        _ptr(labels if head == 0 else None, ctypes.c_int32), _ptr(T if head == 1 else None, ctypes.c_float),
+        ctypes.c_int64(T.shape[1] if head == 1 else 0), ctypes.c_int64(X.shape[0]), ctypes.c_int(head),
+        _ptr(aW, ctypes.c_double), _ptr(ab, ctypes.c_double))
+    assert rc == 0
+    return _unflatten(sizes, aW, ab)
+
+
 def sgd_step(w, g, lr) -> np.ndarray:
     """W - lr*grad evaluated in float64 and rounded once to fp32 (Section 4.2)."""
     w = np.ascontiguousarray(_f32(w)); g = np.ascontiguousarray(_f32(g))

@@ -76,6 +76,29 @@ double oracle_sgemm_entry(int transA, int transB, int64_t K, double alpha,
     return s;
 }
 
+/*
+ * Magnitude sums of the product above: |alpha| * sum_k |op(A)[i][k]| * |op(B)[k][j]| + |beta| * |C_in[i][j]|.
+ * This is the quantity a floating-point evaluation's forward error is proportional to (the error of a sum
+ * is bounded by a multiple of the unit roundoff times the sum of the magnitudes of its terms); the ratio of
+ * its norm to the norm of the product itself is the product's condition number under cancellation.
+ */
+void oracle_sgemm_abs(int transA, int transB, int64_t M, int64_t N, int64_t K, double alpha,
+                      const float* A, int64_t lda, const float* B, int64_t ldb,
+                      double beta, const float* C_in, int64_t ldc, double* out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            double s = 0.0;
+            if (alpha != 0.0) {
+                for (int64_t k = 0; k < K; ++k) s += fabs(opa(A, lda, transA, i, k)) * fabs(opa(B, ldb, !transB, j, k));
+                s *= fabs(alpha);
+            }
+            if (beta != 0.0) s += fabs(beta) * fabs((double)C_in[i * ldc + j]);
+            out[i * N + j] = s;
+        }
+    }
+}
+
 /* ------------------------------------------------------------------------- */
 /* Network description: sizes[0..L], W_l is [sizes[l+1] x sizes[l]] row-major  */
 /* (w_jk: j = unit of the next layer, k = unit of this one, Eqs. 1-2), all W_l */
@@ -170,6 +193,38 @@ static void backward_one(const net_t* n, const float* Wflat, double** act, doubl
                 for (int j = 0; j < nout; ++j) s += (double)W[(int64_t)j * nin + k] * d[j];
                 const double h = act[l][k];
                 delta[l][k] = (1.0 - h * h) * s;
+            }
+        }
+    }
+}
+
+/*
+ * The same back-propagation with every term of every sum taken in absolute value: mag[L] holds the magnitudes
+ * of the output deltas' terms, mag[l][k] = (1 - h^2) * sum_j |w_jk| mag[l+1][j], and the pattern adds
+ * mag[l+1][j] * |act[l][k]| to aW and mag[l+1][j] to ab.  The results bound what rounding errors anywhere in
+ * the evaluation can do to the summed gradient (they are what the errors are proportional to); they are never
+ * smaller than the magnitudes of the gradient's own entries.
+ */
+static void backward_one_abs(const net_t* n, const float* Wflat, double** act, double** mag,
+                             double* aW, double* ab) {
+    for (int l = n->L - 1; l >= 0; --l) {
+        const int nin = n->sizes[l], nout = n->sizes[l + 1];
+        double* aWl = aW + n->woff[l];
+        double* abl = ab + n->boff[l];
+        const double* d = mag[l + 1];
+        for (int j = 0; j < nout; ++j) {
+            const double dj = d[j];
+            abl[j] += dj;
+            double* row = aWl + (int64_t)j * nin;
+            for (int k = 0; k < nin; ++k) row[k] += dj * fabs(act[l][k]);
+        }
+        if (l > 0) {
+            const float* W = Wflat + n->woff[l];
+            for (int k = 0; k < nin; ++k) {
+                double s = 0.0;
+                for (int j = 0; j < nout; ++j) s += fabs((double)W[(int64_t)j * nin + k]) * d[j];
+                const double h = act[l][k];
+                mag[l][k] = (1.0 - h * h) * s;
             }
         }
     }
@@ -285,6 +340,50 @@ int oracle_mlp_probe(int L, const int32_t* sizes, const float* Wflat, const floa
         free(d);
         free_layers(&n, act);
     }
+    return 0;
+}
+
+/*
+ * Magnitude sums of the summed gradient (see backward_one_abs).  head == 0: the output deltas softmax(z) - onehot
+ * enter as softmax(z) + onehot (the subtraction at the label is a cancellation too); head == 1: as |dE/dz|.
+ * aW, ab have the layout of dW, db.
+ */
+int oracle_mlp_gradient_abs(int L, const int32_t* sizes, const float* Wflat, const float* bflat,
+                            const float* X, int64_t ldx, const int32_t* labels, const float* T, int64_t ldt,
+                            int64_t n_patterns, int head, double* aW, double* ab) {
+    net_t n;
+    if (net_init(&n, L, sizes)) return -1;
+    int nthreads = oracle_num_threads();
+    if (nthreads > n_patterns) nthreads = n_patterns > 0 ? (int)n_patterns : 1;
+    double* gW = (double*)calloc((size_t)nthreads * n.nw, sizeof(double));
+    double* gb = (double*)calloc((size_t)nthreads * n.nb, sizeof(double));
+#pragma omp parallel num_threads(nthreads)
+    {
+#ifdef _OPENMP
+        const int t = omp_get_thread_num();
+#else
+        const int t = 0;
+#endif
+        double** act = alloc_layers(&n);
+        double** mag = alloc_layers(&n);
+        const int64_t p0 = n_patterns * t / nthreads, p1 = n_patterns * (t + 1) / nthreads;
+        for (int64_t p = p0; p < p1; ++p) {
+            forward_one(&n, Wflat, bflat, X + p * ldx, act);
+            if (head == 0) {
+                head_softmax_ce(act[L], sizes[L], labels[p], mag[L]);
+                mag[L][labels[p]] += 2.0;                   /* (softmax - 1) + 2 = softmax + 1 */
+            } else {
+                head_tanh_sse(act[L], sizes[L], T + p * ldt, mag[L]);
+                for (int j = 0; j < sizes[L]; ++j) mag[L][j] = fabs(mag[L][j]);
+            }
+            backward_one_abs(&n, Wflat, act, mag, gW + (size_t)t * n.nw, gb + (size_t)t * n.nb);
+        }
+        free_layers(&n, act);
+        free_layers(&n, mag);
+    }
+    for (int64_t i = 0; i < n.nw; ++i) { double s = 0.0; for (int t = 0; t < nthreads; ++t) s += gW[(size_t)t * n.nw + i]; aW[i] = s; }
+    for (int64_t i = 0; i < n.nb; ++i) { double s = 0.0; for (int t = 0; t < nthreads; ++t) s += gb[(size_t)t * n.nb + i]; ab[i] = s; }
+    free(gW); free(gb);
     return 0;
 }
 
