@@ -74,7 +74,14 @@ int ulsnn_version(void);
  * (ulsnn_sgemm_workspace_bytes tells how much; workspace may be NULL when that is 0).  The workspace must be
  * 256-byte aligned and may be reused by the next call on the same stream.
  * Operands that the tensor-core path cannot address with TMA (a base pointer not 16-byte aligned, or a leading
- * dimension that is not a multiple of 4) are computed by the FFMA kernel instead, which is at least as accurate.
+ * dimension that is not a multiple of 4) are first copied into the workspace with their rows padded to a multiple of
+ * four floats (the re-buffering of Section 3.3), and the product then runs on the tensor cores like any other.  The
+ * copies need room: ulsnn_sgemm_workspace_bytes_for, which is given the operands, includes it; ulsnn_sgemm_workspace_bytes,
+ * which is not, covers addressable operands only.  ulsnn_sgemm_ex takes the re-buffered route when the workspace it is
+ * given is large enough for it and computes such a product with the FFMA kernel (at least as accurate, several times
+ * slower) when it is not; C may have any alignment and ldc on either route.
+ * ulsnn_sgemm's own scratch is shared by all its calls on a device: calls on one device must be ordered with respect
+ * to each other (one stream, or events), and any call that needs more scratch than every earlier one may synchronise.
  * ULSNN_MATH_BF16: op(A) and op(B) are first rounded to bfloat16 (round to nearest even) into the workspace, which
  * therefore is never empty in this mode (two bfloat16 copies with rows padded to 8 elements, then the split-K
  * partials); any lda / ldb is accepted.  C, alpha and beta stay fp32.  Expect a relative error of about 2e-3.
@@ -89,6 +96,11 @@ ulsnn_status_t ulsnn_sgemm_ex(char transA, char transB, int64_t M, int64_t N, in
                               void* workspace, size_t workspace_bytes, ulsnn_stream_t stream);
 ulsnn_status_t ulsnn_sgemm_workspace_bytes(char transA, char transB, int64_t M, int64_t N, int64_t K,
                                            ulsnn_math_t math, size_t* bytes /* host, out */);
+/* The same for given operands: A, B (device pointers, inspected for their alignment only, never read) and their leading
+ * dimensions.  Includes the room for re-buffered copies of operands TMA cannot address (Section 3.3). */
+ulsnn_status_t ulsnn_sgemm_workspace_bytes_for(char transA, char transB, int64_t M, int64_t N, int64_t K,
+                                               const float* A, int64_t lda, const float* B, int64_t ldb,
+                                               ulsnn_math_t math, size_t* bytes /* host, out */);
 
 /*
  * SGEMM for callers that cannot allocate device memory (the paper has no counterpart of this call).
@@ -100,8 +112,11 @@ ulsnn_status_t ulsnn_sgemm_workspace_bytes(char transA, char transB, int64_t M, 
  * the same `math`, but takes its split-K scratch from a fixed array of ulsnn_sgemm_noalloc_max_scratch_bytes()
  * (8 MiB) that is part of the library's image on every GPU that loads it.  It calls neither cudaMalloc nor
  * cudaFree nor any allocating routine.
- *  - A product whose split-K partials do not fit (ulsnn_sgemm_workspace_bytes(...) > the maximum) is rejected
- *    with ULSNN_ERR_TOO_LARGE and nothing is launched.  Products that need no split never touch the array.
+ *  - A product whose scratch does not fit is rejected with ULSNN_ERR_TOO_LARGE and nothing is launched.  What is
+ *    compared with the maximum is the scratch the product actually needs on the route it takes (split-K partials;
+ *    in ULSNN_MATH_BF16 also the two bfloat16 copies; for operands TMA cannot address their re-buffered copies when
+ *    those fit, else the FFMA kernel's partials), which can be less than ulsnn_sgemm_workspace_bytes reports.
+ *    Products that need no scratch never touch the array.
  *  - The first call on each device that needs the array looks up the array's device address (with that device
  *    current); make that first call outside any stream capture.
  *  - All calls on a device share the one array, and it keeps the previous call's contents (nothing has to start
@@ -197,8 +212,9 @@ ulsnn_status_t ulsnn_vec_dot(int64_t n, const float* x, const float* y, double* 
                              size_t workspace_bytes, ulsnn_stream_t stream);
 ulsnn_status_t ulsnn_vec_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out,
                                ulsnn_stream_t stream);
-/* Synchronises `stream`, then returns ULSNN_OK, ULSNN_ERR_DEVICE_TIMEOUT if a kernel of this handle gave up a
- * bounded wait since the last call of this function (the word is cleared), or ULSNN_ERR_CUDA. */
+/* Synchronises `stream`, then returns ULSNN_OK, ULSNN_ERR_DEVICE_TIMEOUT if any kernel of the library gave up a
+ * bounded wait on the current device since the last call of this function there (the status word belongs to the
+ * device, not to the handle, which may be NULL; the call clears it), or ULSNN_ERR_CUDA. */
 ulsnn_status_t ulsnn_last_device_status(ulsnn_mlp_t* handle, ulsnn_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
@@ -232,6 +248,19 @@ void ulsnn_launch_counts(int64_t counts[4]);
  */
 ulsnn_status_t ulsnn_mlp_enable_timing(ulsnn_mlp_t* handle, int on);
 ulsnn_status_t ulsnn_mlp_phase_times(ulsnn_mlp_t* handle, int* n, float* ms, int64_t* mnk);
+/*
+ * Checks of the library's own safety net (no counterpart in the paper).
+ * ulsnn_debug_wait_timeout: enqueues one thread block that allocates tensor memory as the product kernels do and then
+ *   waits on a barrier nothing ever arrives on, with a limit of limit_cycles SM clock cycles (1 .. 2e9).  The wait runs
+ *   out, the block records the time-out in the device status word, frees its tensor memory and returns by itself; the
+ *   next ulsnn_last_device_status() on the device returns ULSNN_ERR_DEVICE_TIMEOUT.  Nothing traps or faults, and
+ *   the context stays usable.  This is the path every bounded wait of the product kernels takes when it gives up.
+ * ulsnn_debug_device_cache_slot: the slot of a device ordinal in the library's per-device host tables (architecture
+ *   check, SM count, symbol addresses, kernel attributes, scratch buffers), or -1 when the ordinal is outside them
+ *   (such a device is refused).  Host only.
+ */
+ulsnn_status_t ulsnn_debug_wait_timeout(uint64_t limit_cycles, ulsnn_stream_t stream);
+int            ulsnn_debug_device_cache_slot(int device);
 
 #ifdef __cplusplus
 }

@@ -199,6 +199,46 @@ def mlp_gradient_abs(Ws, bs, X, labels=None, T=None):
     return _unflatten(sizes, aW, ab)
 
 
+def perturb_inputs(Ws, bs, X, T=None, eps=2.0 ** -14, seed=0):
+    """Copies of the parameters, the patterns and (if given) the dense targets with every entry multiplied by
+    1 + eps*u, u uniform in [-1, 1) from numpy's default_rng(seed), drawn tensor by tensor in the order
+    W_0.., b_0.., X, T, evaluated in float64 and rounded to fp32.  Labels are not perturbed."""
+    rng = np.random.default_rng(seed)
+
+    def pert(a):
+        a = _f32(a)
+        return (a.astype(np.float64) * (1.0 + eps * rng.uniform(-1.0, 1.0, a.shape))).astype(np.float32)
+
+    Wp = [pert(w) for w in Ws]
+    bp = [pert(b) for b in bs]
+    Xp = pert(X)
+    Tp = pert(T) if T is not None else None
+    return Wp, bp, Xp, Tp
+
+
+def gradient_condition(Ws, bs, X, labels=None, T=None, eps=2.0 ** -14, seeds=(12345, 12346)):
+    """Estimated relative condition number of every tensor of the summed gradient with respect to componentwise
+    relative perturbations of its inputs: ||g(inputs*(1+eta)) - g(inputs)||_2 / ||g(inputs)||_2 divided by the
+    root-mean-square size eps/sqrt(3) of the random eta, the larger of the values of the given seeds.
+    Returns ([cond dW_l], [cond db_l]).  A finite-precision evaluation commits relative errors of the size of its
+    unit roundoff in inputs and intermediates, so its attainable relative error is proportional to this number."""
+    def grad(Wq, bq, Xq, Tq):
+        return mlp_gradient(Wq, bq, Xq, labels) if T is None else mlp_sse_gradient(Wq, bq, Xq, Tq)
+
+    _, gW, gb = grad(Ws, bs, X, T)
+    rms = eps / np.sqrt(3.0)
+    best = None
+    for seed in seeds:
+        Wp, bp, Xp, Tp = perturb_inputs(Ws, bs, X, T, eps, seed)
+        _, pW, pb = grad(Wp, bp, Xp, Tp)
+        c = []
+        for a, b in zip(pW + pb, gW + gb):
+            r = np.linalg.norm(b.ravel())
+            c.append(float(np.linalg.norm((a - b).ravel()) / r / rms) if r > 0 else 0.0)
+        best = c if best is None else [max(u, v) for u, v in zip(best, c)]
+    return best[:len(Ws)], best[len(Ws):]
+
+
 def sgd_step(w, g, lr) -> np.ndarray:
     """W - lr*grad evaluated in float64 and rounded once to fp32 (Section 4.2)."""
     w = np.ascontiguousarray(_f32(w)); g = np.ascontiguousarray(_f32(g))

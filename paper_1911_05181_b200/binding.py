@@ -33,6 +33,7 @@ EXPORTS = [
     "ulsnn_fill_labels", "ulsnn_launch_counts", "ulsnn_mlp_enable_timing", "ulsnn_mlp_phase_times",
     "ulsnn_sgemm_noalloc", "ulsnn_sgemm_noalloc_max_scratch_bytes", "ulsnn_mlp_forward_sse", "ulsnn_mlp_gradient_sse",
     "ulsnn_vec_dot_workspace_bytes", "ulsnn_vec_dot", "ulsnn_vec_axpby",
+    "ulsnn_sgemm_workspace_bytes_for", "ulsnn_debug_wait_timeout", "ulsnn_debug_device_cache_slot",
 ]
 
 
@@ -69,6 +70,11 @@ def lib():
         l.ulsnn_sgemm_noalloc_max_scratch_bytes.argtypes = []
         l.ulsnn_sgemm_workspace_bytes.argtypes = [ctypes.c_char, ctypes.c_char, i64, i64, i64, ctypes.c_int,
                                                   ctypes.POINTER(sz)]
+        l.ulsnn_sgemm_workspace_bytes_for.argtypes = [ctypes.c_char, ctypes.c_char, i64, i64, i64, vp, i64, vp, i64,
+                                                      ctypes.c_int, ctypes.POINTER(sz)]
+        l.ulsnn_debug_wait_timeout.argtypes = [u64, vp]
+        l.ulsnn_debug_device_cache_slot.argtypes = [ctypes.c_int]
+        l.ulsnn_debug_device_cache_slot.restype = ctypes.c_int
         l.ulsnn_mlp_workspace_bytes.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(sz)]
         l.ulsnn_mlp_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(_Desc), vp, sz]
         l.ulsnn_mlp_destroy.argtypes = [vp]
@@ -147,6 +153,27 @@ def sgemm_workspace_bytes(transA, transB, M, N, K, math=MATH_3XTF32) -> int:
     _check(lib().ulsnn_sgemm_workspace_bytes(transA.encode(), transB.encode(), M, N, K, math, ctypes.byref(out)),
            "ulsnn_sgemm_workspace_bytes")
     return out.value
+
+
+def sgemm_workspace_bytes_for(transA, transB, M, N, K, A, lda, B, ldb, math=MATH_3XTF32) -> int:
+    """Workspace for these operands (A, B: tensors or addresses, inspected for alignment only)."""
+    out = ctypes.c_size_t(0)
+    _check(lib().ulsnn_sgemm_workspace_bytes_for(transA.encode(), transB.encode(), M, N, K, _ptr(A), lda, _ptr(B), ldb,
+                                                 math, ctypes.byref(out)), "ulsnn_sgemm_workspace_bytes_for")
+    return out.value
+
+
+def debug_wait_timeout(limit_cycles: int, stream=None) -> int:
+    return lib().ulsnn_debug_wait_timeout(int(limit_cycles), _stream(stream))
+
+
+def device_cache_slot(device: int) -> int:
+    return int(lib().ulsnn_debug_device_cache_slot(int(device)))
+
+
+def last_device_status(stream=None) -> int:
+    """Status word of the current device (synchronises the stream, clears the word)."""
+    return lib().ulsnn_last_device_status(None, _stream(stream))
 
 
 def sgemm_ex(transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, math=MATH_3XTF32,

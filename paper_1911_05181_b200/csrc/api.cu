@@ -29,10 +29,10 @@ bool parse_trans(char c, bool* t) {
 
 ulsnn_status_t check_arch() {
     static std::mutex mu;
-    static int cached[64];          // 0 unknown, 1 ok, 2 unsupported
+    static int cached[MAX_DEVICE_SLOTS];          // 0 unknown, 1 ok, 2 unsupported
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ULSNN_ERR_CUDA;
-    if (dev < 0 || dev >= 64) return ULSNN_ERR_UNSUPPORTED_ARCH;
+    if (device_cache_slot(dev) < 0) return ULSNN_ERR_UNSUPPORTED_ARCH;
     std::lock_guard<std::mutex> lk(mu);
     if (cached[dev] == 0) {
         int major = 0;
@@ -114,15 +114,71 @@ size_t sgemm_ws_for(const GemmDesc& d, bool tc) {
 
 ulsnn_status_t half_sgemm_impl(const SgemmArgs& a, void* ws, size_t ws_bytes, cudaStream_t stream);
 
-ulsnn_status_t sgemm_impl(const SgemmArgs& a, ulsnn_math_t math, void* ws, size_t ws_bytes, cudaStream_t stream) {
-    if (a.M == 0 || a.N == 0) return ULSNN_OK;
-    if (!a.C) return ULSNN_ERR_INVALID_ARG;
-    if (a.K == 0 || a.alpha == 0.f) {
-        if (a.beta == 1.f) return ULSNN_OK;
-        return launch_scale_rows(a.C, a.M, a.N, a.ldc, a.beta, stream);
+// Re-buffering of operands the tensor-core path cannot address with TMA (Section 3.3 copies B' into a buffer laid out
+// for the kernel): an operand whose base is not 16-byte aligned or whose leading dimension is not a multiple of 4 is
+// copied into the workspace with its rows padded to a multiple of four floats; the product then runs on the tensor
+// cores as for any other operand.  The workspace holds [copy of A][copy of B][split-K partials].
+struct PackPlan {
+    bool a, b;                      // which operands are copied
+    int64_t a_rows, a_cols, lda, b_rows, b_cols, ldb;
+    size_t a_bytes, b_bytes;
+};
+
+PackPlan pack_plan(const SgemmArgs& a) {
+    PackPlan pl{};
+    pl.a_rows = a.ta ? a.K : a.M; pl.a_cols = a.ta ? a.M : a.K; pl.lda = round_up(pl.a_cols, 4);
+    pl.b_rows = a.tb ? a.N : a.K; pl.b_cols = a.tb ? a.K : a.N; pl.ldb = round_up(pl.b_cols, 4);
+    pl.a = !tc_operand_addressable(a.A, a.lda);
+    pl.b = !tc_operand_addressable(a.B, a.ldb);
+    pl.a_bytes = pl.a ? align256((size_t)pl.a_rows * pl.lda * sizeof(float)) : 0;
+    pl.b_bytes = pl.b ? align256((size_t)pl.b_rows * pl.ldb * sizeof(float)) : 0;
+    return pl;
+}
+
+// the product with its re-buffered operands at `ws`
+SgemmArgs packed_args(const SgemmArgs& a, const PackPlan& pl, void* ws) {
+    SgemmArgs t = a;
+    if (pl.a) { t.A = (const float*)ws; t.lda = pl.lda; }
+    if (pl.b) { t.B = (const float*)((char*)ws + pl.a_bytes); t.ldb = pl.ldb; }
+    return t;
+}
+
+// Scratch the re-buffered tensor-core route needs for these operands (0 when they need no re-buffering or the route
+// does not exist for them).
+size_t sgemm_packed_need(const SgemmArgs& a, ulsnn_math_t math) {
+    if (math != ULSNN_MATH_3XTF32 && math != ULSNN_MATH_TF32) return 0;
+    const PackPlan pl = pack_plan(a);
+    if (!pl.a && !pl.b) return 0;
+    // a stand-in address with the alignment the copies will have
+    const SgemmArgs t = packed_args(a, pl, (void*)(uintptr_t)256);
+    const GemmDesc d = sgemm_desc(t);
+    if (!tc_gemm_supported(d)) return 0;
+    return pl.a_bytes + pl.b_bytes + sgemm_ws_for(d, true);
+}
+
+ulsnn_status_t sgemm_impl(const SgemmArgs& a_in, ulsnn_math_t math, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    if (a_in.M == 0 || a_in.N == 0) return ULSNN_OK;
+    if (!a_in.C) return ULSNN_ERR_INVALID_ARG;
+    if (a_in.K == 0 || a_in.alpha == 0.f) {
+        if (a_in.beta == 1.f) return ULSNN_OK;
+        return launch_scale_rows(a_in.C, a_in.M, a_in.N, a_in.ldc, a_in.beta, stream);
     }
-    if (!a.A || !a.B) return ULSNN_ERR_INVALID_ARG;
-    if (math == ULSNN_MATH_BF16) return half_sgemm_impl(a, ws, ws_bytes, stream);
+    if (!a_in.A || !a_in.B) return ULSNN_ERR_INVALID_ARG;
+    if (math == ULSNN_MATH_BF16) return half_sgemm_impl(a_in, ws, ws_bytes, stream);
+    SgemmArgs a = a_in;
+    if (!use_tc(sgemm_desc(a), math)) {
+        // the re-buffered route, when the workspace has room for it; otherwise the FFMA kernel takes the operands as they are
+        const size_t need = sgemm_packed_need(a, math);
+        if (need > 0 && ws && ws_bytes >= need && ((uintptr_t)ws & 255) == 0) {
+            const PackPlan pl = pack_plan(a);
+            a = packed_args(a_in, pl, ws);
+            ulsnn_status_t st = ULSNN_OK;
+            if (pl.a && (st = launch_pack_rows(a_in.A, pl.a_rows, pl.a_cols, a_in.lda, (float*)a.A, pl.lda, stream)) != ULSNN_OK) return st;
+            if (pl.b && (st = launch_pack_rows(a_in.B, pl.b_rows, pl.b_cols, a_in.ldb, (float*)a.B, pl.ldb, stream)) != ULSNN_OK) return st;
+            ws = (char*)ws + pl.a_bytes + pl.b_bytes;
+            ws_bytes -= pl.a_bytes + pl.b_bytes;
+        }
+    }
     GemmDesc d = sgemm_desc(a);
     const bool tc = use_tc(d, math);
     const SplitPlan p = plan_splits(tiles_of(d, tc), d.K, slots_of(d, tc));
@@ -195,9 +251,11 @@ size_t sgemm_need(const SgemmArgs& a, ulsnn_math_t math) {
     return sgemm_ws_for(d, use_tc(d, math));
 }
 
-// grow-only scratch of ulsnn_sgemm, one per device
-struct DevScratch { void* p = nullptr; size_t bytes = 0; };
-DevScratch g_scratch[64];
+// Scratch of ulsnn_sgemm, one per device.  It only grows, and a buffer that has been handed to a call is never freed
+// before the process exits (a larger one is allocated beside it): a product enqueued by another host thread may still
+// be reading it.
+struct DevScratch { void* p = nullptr; size_t bytes = 0; std::vector<void*> retired; };
+DevScratch g_scratch[MAX_DEVICE_SLOTS];
 std::mutex g_scratch_mu;
 
 }  // namespace
@@ -220,7 +278,7 @@ extern "C" const char* ulsnn_status_string(ulsnn_status_t s) {
     return "unknown status";
 }
 
-extern "C" int ulsnn_version(void) { return 108; }
+extern "C" int ulsnn_version(void) { return 109; }
 
 extern "C" void ulsnn_launch_counts(int64_t counts[4]) {
     for (int i = 0; i < 4; ++i) counts[i] = g_counts[i].load(std::memory_order_relaxed);
@@ -241,6 +299,23 @@ extern "C" ulsnn_status_t ulsnn_sgemm_workspace_bytes(char transA, char transB, 
     GemmDesc d = sgemm_desc(a);
     size_t w = sgemm_ws_for(d, false);
     if (math != ULSNN_MATH_FP32_SIMT) { const size_t w2 = sgemm_ws_for(d, true); if (w2 > w) w = w2; }
+    *bytes = w;
+    return ULSNN_OK;
+}
+
+extern "C" ulsnn_status_t ulsnn_sgemm_workspace_bytes_for(char transA, char transB, int64_t M, int64_t N, int64_t K,
+                                                          const float* A, int64_t lda, const float* B, int64_t ldb,
+                                                          ulsnn_math_t math, size_t* bytes) {
+    SgemmArgs a{false, false, M, N, K, 1.f, 0.f, A, lda, B, ldb, nullptr, N > 1 ? N : 1};
+    if (!bytes) return ULSNN_ERR_INVALID_ARG;
+    ulsnn_status_t st = validate_sgemm(transA, transB, M, N, K, lda, ldb, a.ldc, &a.ta, &a.tb);
+    if (st != ULSNN_OK) return st;
+    if ((int)math < 0 || (int)math > 3) return ULSNN_ERR_INVALID_ARG;
+    *bytes = 0;
+    if (M == 0 || N == 0 || K == 0) return ULSNN_OK;
+    size_t w = sgemm_need(a, math);
+    const size_t packed = sgemm_packed_need(a, math);
+    if (packed > w) w = packed;
     *bytes = w;
     return ULSNN_OK;
 }
@@ -269,17 +344,18 @@ extern "C" ulsnn_status_t ulsnn_sgemm(char transA, char transB, int64_t M, int64
     void* ws = nullptr; size_t have = 0;
     if (K > 0 && alpha != 0.f && A && B && C) {
         GemmDesc d = sgemm_desc(a);
-        const size_t need = sgemm_ws_for(d, use_tc(d, ULSNN_MATH_3XTF32));
+        size_t need = sgemm_ws_for(d, use_tc(d, ULSNN_MATH_3XTF32));
+        const size_t packed = sgemm_packed_need(a, ULSNN_MATH_3XTF32);
+        if (packed > need) need = packed;
         int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ULSNN_ERR_CUDA;
+        if (cudaGetDevice(&dev) != cudaSuccess || device_cache_slot(dev) < 0) return ULSNN_ERR_CUDA;
         std::lock_guard<std::mutex> lk(g_scratch_mu);
-        DevScratch& sc = g_scratch[dev];
+        DevScratch& sc = g_scratch[device_cache_slot(dev)];
         if (need > sc.bytes) {
-            // cudaFree waits for all work on the device, so nothing still reads the old buffer
-            if (sc.p) cudaFree(sc.p);
-            sc.p = nullptr; sc.bytes = 0;
-            if (cudaMalloc(&sc.p, need) != cudaSuccess) { sc.p = nullptr; return ULSNN_ERR_CUDA; }
-            sc.bytes = need;
+            void* bigger = nullptr;
+            if (cudaMalloc(&bigger, need) != cudaSuccess) return ULSNN_ERR_CUDA;
+            if (sc.p) sc.retired.push_back(sc.p);
+            sc.p = bigger; sc.bytes = need;
         }
         ws = sc.p; have = sc.bytes;
     }
@@ -298,11 +374,11 @@ namespace {
 // In host code `g_noalloc_scratch` is only a handle of the symbol; the address a kernel can use has to be asked for,
 // per device, with that device current.
 std::mutex g_noalloc_mu;
-void* g_noalloc_ptr[64];
+void* g_noalloc_ptr[MAX_DEVICE_SLOTS];
 
 ulsnn_status_t noalloc_scratch(void** out) {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ULSNN_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || device_cache_slot(dev) < 0) return ULSNN_ERR_CUDA;
     std::lock_guard<std::mutex> lk(g_noalloc_mu);
     if (!g_noalloc_ptr[dev]) {
         void* p = nullptr;
@@ -328,8 +404,12 @@ extern "C" ulsnn_status_t ulsnn_sgemm_noalloc(char transA, char transB, int64_t 
     if (M == 0 || N == 0) return ULSNN_OK;
     size_t need = 0;
     if (K > 0 && alpha != 0.f && A && B && C) {
-        // the same slice plan as ulsnn_sgemm_ex makes for these operands, so the two give the same bits
+        // the same route and slice plan as ulsnn_sgemm_ex takes for these operands when it is given the workspace
+        // ulsnn_sgemm_workspace_bytes_for asks for, so the two give the same bits: operands TMA cannot address are
+        // re-buffered in the array when copies and partials fit, and go to the FFMA kernel when they do not
         need = sgemm_need(a, math);
+        const size_t packed = sgemm_packed_need(a, math);
+        if (packed > need && packed <= (size_t)ULSNN_NOALLOC_SCRATCH_BYTES) need = packed;
     }
     if (need > (size_t)ULSNN_NOALLOC_SCRATCH_BYTES) return ULSNN_ERR_TOO_LARGE;
     if ((st = check_arch()) != ULSNN_OK) return st;
@@ -937,8 +1017,17 @@ extern "C" ulsnn_status_t ulsnn_vec_axpby(int64_t n, float a, const float* x, fl
     return launch_axpby(n, a, x, b, y, out, (cudaStream_t)stream);
 }
 
+extern "C" int ulsnn_debug_device_cache_slot(int device) { return device_cache_slot(device); }
+
+extern "C" ulsnn_status_t ulsnn_debug_wait_timeout(uint64_t limit_cycles, ulsnn_stream_t stream) {
+    if (limit_cycles == 0 || limit_cycles > 2000000000ull) return ULSNN_ERR_INVALID_ARG;
+    ulsnn_status_t st = check_arch();
+    if (st != ULSNN_OK) return st;
+    return tc_wait_probe_launch((unsigned long long)limit_cycles, (cudaStream_t)stream);
+}
+
 extern "C" ulsnn_status_t ulsnn_last_device_status(ulsnn_mlp_t* h, ulsnn_stream_t stream) {
-    (void)h;
+    (void)h;        // the status word belongs to the device, not to a handle
     int word = 0;
     ulsnn_status_t st = device_status_fetch_and_clear((cudaStream_t)stream, &word);
     if (st != ULSNN_OK) return st;

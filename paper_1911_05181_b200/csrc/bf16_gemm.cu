@@ -47,7 +47,6 @@ constexpr int EPI_STAGE_BYTES = 32 * 128;           // one block of 32 rows x 12
 constexpr int EPI_BUFS = 1;
 constexpr int EPI_SCRATCH_BYTES = NUM_EPI_WARPS * EPI_BUFS * EPI_STAGE_BYTES;
 constexpr int CTRL_BYTES = 1024;
-constexpr unsigned long long WAIT_LIMIT_CYCLES = 3000000000ull;
 constexpr float LOG2E = 1.4426950408889634f;
 
 struct HgParams {
@@ -55,6 +54,7 @@ struct HgParams {
     int bn, n_gran, tiles_m, tiles_n, units, stages, b_tile_bytes, stage_bytes;
     int a_mn, b_mn;
     int c_tma;
+    unsigned long long wait_limit;      // clock cycles a device-side wait may take before the CTA gives up
     int* status;
 };
 
@@ -66,29 +66,8 @@ struct Ctrl {
     uint64_t free_sink[2][NUM_EPI_WARPS];
     uint32_t tmem_base;
     volatile int abort;
+    unsigned long long wait_limit;
 };
-
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctrl* ctrl, int* status) {
-    const uint32_t b = smem_u32(bar);
-    if (mbar_try_wait(b, parity)) return true;
-    const unsigned long long t0 = clock64();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(b, parity)) {
-        if ((++spins & 255u) == 0) {
-            if (ctrl->abort) return false;
-            if ((unsigned long long)clock64() - t0 > WAIT_LIMIT_CYCLES) {
-                ctrl->abort = 1;
-                atomicExch(status, DEV_TIMEOUT);
-                return false;
-            }
-        }
-    }
-    return true;
-}
-__device__ __forceinline__ bool wait_bar_warp(uint64_t* bar, uint32_t parity, Ctrl* ctrl, int* status) {
-    const bool ok = wait_bar(bar, parity, ctrl, status);
-    return __all_sync(0xffffffffu, ok);
-}
 
 template <int CG>
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -123,26 +102,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-__device__ __forceinline__ void unit_coords(const HgParams& p, int u, int& mt, int& nt, int& sp) {
-    nt = u % p.tiles_n;
-    const int r = u / p.tiles_n;
-    mt = r % p.tiles_m;
-    sp = r / p.tiles_m;
-}
-__device__ __forceinline__ int tile_cols(const HgParams& p, int nt) {
-    const int left = (int)p.d.N - nt * p.bn;
-    return left >= p.bn ? p.bn : (left + p.n_gran - 1) / p.n_gran * p.n_gran;
-}
-__device__ __forceinline__ void unit_k_range(const HgParams& p, int sp, int64_t& kbeg, int& nkb, int& tail_steps) {
-    kbeg = (p.d.epi == EPI_PARTIAL) ? (int64_t)sp * p.d.k_per_split : 0;
-    int64_t kend = (p.d.epi == EPI_PARTIAL) ? kbeg + p.d.k_per_split : p.d.K;
-    if (kend > p.d.K) kend = p.d.K;
-    const int64_t len = kend - kbeg;
-    nkb = (int)((len + BK - 1) / BK);
-    const int rem = (int)(len - (int64_t)(nkb - 1) * BK);
-    tail_steps = (rem + UMMA_K - 1) / UMMA_K;
-}
-
 template <int EPI, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -170,6 +129,7 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             mbar_init(smem_u32(&ctrl->reg_free[a]), NUM_EPI_WARPS + (CG == 2 ? 1 : 0));
         }
         ctrl->abort = 0;
+        ctrl->wait_limit = p.wait_limit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -189,7 +149,7 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         bool ok = true;
         for (int u = first_unit; u < p.units && ok; u += unit_step) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-            int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+            int64_t kbeg; int nkb, tail; unit_k_range<BK, UMMA_K>(p, sp, kbeg, nkb, tail);
             const int b_cols = tile_cols(p, nt) / CG;
             const int m0 = (mt * CG + rank) * BM, n0 = nt * p.bn + rank * b_cols;
             const int b_boxes = b_cols >> 6;        // MN-major B: boxes of 64 columns, only those the products read
@@ -251,7 +211,7 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             bool ok = true;
             for (int u = first_unit; u < p.units && ok; u += unit_step, ++tile_i) {
                 int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-                int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+                int64_t kbeg; int nkb, tail; unit_k_range<BK, UMMA_K>(p, sp, kbeg, nkb, tail);
                 const uint32_t idesc = idesc0 | ((uint32_t)(tile_cols(p, nt) >> 3) << 17);
                 const uint32_t reg = tile_i & 1;
                 if (tile_i >= 2) {      // the region has held a tile before: wait until every epilogue warp has read it
@@ -661,25 +621,13 @@ bool operand_ok(const void* base, int64_t ld) {
     return (((uintptr_t)base) & 15) == 0 && (ld & 7) == 0 && ld >= 8 && ld < ((int64_t)1 << 38);
 }
 
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = NUM_SMS;
-    }
-    return n;
-}
+int sm_count() { return sm_count_of_current_device(NUM_SMS); }
 
 template <int EPI, int CG>
 ulsnn_status_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const HgParams& p, int smem_bytes,
                       int grid, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(bf16_gemm_kernel<EPI, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
-            return ULSNN_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<uint64_t> configured{0};
+    if (!allow_dynamic_smem(bf16_gemm_kernel<EPI, CG>, SMEM_BUDGET, configured)) return ULSNN_ERR_CUDA;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
     cfg.blockDim = dim3(NUM_THREADS, 1, 1);
@@ -753,6 +701,7 @@ ulsnn_status_t hg_gemm_launch(const HalfGemmDesc& d, cudaStream_t stream) {
     if (stages < 2) return ULSNN_ERR_INVALID_ARG;
     p.stages = stages;
     p.status = device_status_word();
+    p.wait_limit = DEFAULT_WAIT_LIMIT_CYCLES;
     if (!p.status) return ULSNN_ERR_CUDA;
 
     CUtensorMap ma, mb, mc;

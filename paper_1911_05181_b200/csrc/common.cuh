@@ -82,6 +82,11 @@ struct HalfGemmDesc {
 // Device status word values (0 = fine).
 enum : int { DEV_OK = 0, DEV_TIMEOUT = 1 };
 
+// Host-side caches of per-device facts (architecture check, SM count, symbol addresses, kernel attributes, scratch
+// buffers) are arrays indexed by this slot: the device ordinal, or -1 when it is outside the table.
+constexpr int MAX_DEVICE_SLOTS = 64;
+inline int device_cache_slot(int device) { return (device >= 0 && device < MAX_DEVICE_SLOTS) ? device : -1; }
+
 // engines
 ulsnn_status_t simt_gemm_launch(const GemmDesc& d, cudaStream_t stream);
 int simt_tile_m();
@@ -99,7 +104,10 @@ int tc_colsum_groups();
 int simt_colsum_groups();
 ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stream);
 // device status word shared by all kernels of the library on the current device
-int* device_status_word();      // its device address (null if it cannot be had)
+int* device_status_word();      // its address on the current device (null if it cannot be had)
+// One CTA that waits, with the given limit in clock cycles, on a barrier nothing ever arrives on: the wait runs out,
+// the CTA records DEV_TIMEOUT, frees its tensor memory and returns.  For the test of the bounded-wait path.
+ulsnn_status_t tc_wait_probe_launch(unsigned long long limit_cycles, cudaStream_t stream);
 ulsnn_status_t device_status_fetch_and_clear(cudaStream_t stream, int* word);
 
 // 16-bit tcgen05 engine (bf16_gemm.cu): operands need 16-byte aligned bases and leading dimensions that are
@@ -161,6 +169,11 @@ ulsnn_status_t launch_sgd_multi(const SgdBatch& b, float lr, cudaStream_t stream
 ulsnn_status_t launch_zero(float* p, int64_t n, cudaStream_t stream);
 ulsnn_status_t launch_zero_f64(double* p, int64_t n, cudaStream_t stream);
 ulsnn_status_t launch_scale_rows(float* C, int64_t M, int64_t N, int64_t ldc, float beta, cudaStream_t stream);
+// dst[r][c] = src[r][c] (c < cols), 0 for cols <= c < ldd; dst 16-byte aligned, ldd a multiple of 4
+ulsnn_status_t launch_pack_rows(const float* src, int64_t rows, int64_t cols, int64_t lds, float* dst, int64_t ldd,
+                                cudaStream_t stream);
+// can TMA address a row-major fp32 operand with this base and leading dimension?
+bool tc_operand_addressable(const float* base, int64_t ld);
 
 // launch accounting: kind 0 FFMA GEMM, 1 tcgen05 GEMM, 2 reductions/small kernels, 3 fills
 void count_launch(int kind);

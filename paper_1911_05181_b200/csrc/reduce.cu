@@ -429,6 +429,40 @@ ulsnn_status_t launch_zero_f64(double* p, int64_t n, cudaStream_t stream) {
     return cuda_ok(cudaGetLastError());
 }
 
+// Re-buffering of an operand the tensor-core path cannot address (Section 3.3 copies B' into a buffer laid out for
+// the kernel; here the reason is TMA's need for 16-byte aligned rows): dst[r][c] = src[r][c] for c < cols, 0 in the
+// padding up to ldd (a multiple of 4).  One warp per 128-column piece of a row, rows strided over the grid; the reads
+// are 4-byte (the source rows are not aligned), the writes 16-byte.
+__global__ void pack_rows_kernel(const float* __restrict__ src, int64_t rows, int64_t cols, int64_t lds,
+                                 float* __restrict__ dst, int64_t ldd) {
+    const int lane = threadIdx.x & 31;
+    const int64_t pieces = (ldd + 127) / 128;
+    const int64_t total = rows * pieces;
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); w < total; w += warps) {
+        const int64_t r = w / pieces, c0 = (w % pieces) * 128 + 4 * lane;
+        if (c0 >= ldd) continue;
+        const float* s = src + r * lds + c0;
+        float4 v;
+        v.x = c0 + 0 < cols ? __ldg(s + 0) : 0.f;
+        v.y = c0 + 1 < cols ? __ldg(s + 1) : 0.f;
+        v.z = c0 + 2 < cols ? __ldg(s + 2) : 0.f;
+        v.w = c0 + 3 < cols ? __ldg(s + 3) : 0.f;
+        *reinterpret_cast<float4*>(dst + r * ldd + c0) = v;
+    }
+}
+
+ulsnn_status_t launch_pack_rows(const float* src, int64_t rows, int64_t cols, int64_t lds, float* dst, int64_t ldd,
+                                cudaStream_t stream) {
+    if (rows <= 0 || cols <= 0) return ULSNN_OK;
+    const int64_t pieces = rows * ((ldd + 127) / 128);
+    int64_t blocks = (pieces + 7) / 8;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    pack_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(src, rows, cols, lds, dst, ldd);
+    ulsnn::count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
 ulsnn_status_t launch_scale_rows(float* C, int64_t M, int64_t N, int64_t ldc, float beta, cudaStream_t stream) {
     if (M <= 0 || N <= 0) return ULSNN_OK;
     scale_rows_kernel<<<grid_for(M * N, 256), 256, 0, stream>>>(C, M, N, ldc, beta);

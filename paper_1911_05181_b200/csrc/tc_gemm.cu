@@ -35,6 +35,7 @@
 #include <cuda.h>
 #include <math.h>
 #include <string.h>
+#include <atomic>
 #include <mutex>
 #include <type_traits>
 
@@ -66,7 +67,6 @@ constexpr int SMEM_BUDGET = 227 * 1024;
 constexpr int EPI_STAGE_BYTES = 32 * 128;                        // one 32x32 fp32 block, 128B-swizzled
 constexpr int EPI_SCRATCH_BYTES = NUM_EPI_WARPS * 2 * EPI_STAGE_BYTES;   // two store-staging blocks per epilogue warp
 constexpr int CTRL_BYTES = 1024;                                // barriers, TMEM base, abort flag
-constexpr unsigned long long WAIT_LIMIT_CYCLES = 3000000000ull; // ~1.5 s at 2 GHz
 
 struct TcParams {
     GemmDesc d;
@@ -87,6 +87,7 @@ struct TcParams {
     int direct;             // CTA pairs without an operand pass: both CTAs count their landed bytes on CTA 0's `full`
                             // barriers (cta_group::2 loads), nothing is relayed
     int64_t n_patterns, n_classes;      // bounds of the logits operand when a_transform
+    unsigned long long wait_limit;      // clock cycles a device-side wait may take before the CTA gives up
     int* status;
 };
 
@@ -100,55 +101,8 @@ struct Ctrl {
     uint64_t free_sink[2][NUM_EPI_WARPS];   // CTA 0: landing words of CTA 1's accumulator-free signals
     uint32_t tmem_base;
     volatile int abort;
+    unsigned long long wait_limit;
 };
-
-// Bounded wait.  Returns false (after raising the abort flag and the device status) if the phase did not complete.
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctrl* ctrl, int* status) {
-    const uint32_t b = smem_u32(bar);
-    if (mbar_try_wait(b, parity)) return true;
-    const unsigned long long t0 = clock64();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(b, parity)) {
-        if ((++spins & 255u) == 0) {
-            if (ctrl->abort) return false;
-            if ((unsigned long long)clock64() - t0 > WAIT_LIMIT_CYCLES) {
-                ctrl->abort = 1;
-                atomicExch(status, DEV_TIMEOUT);
-                return false;
-            }
-        }
-    }
-    return true;
-}
-
-// wait_bar by all lanes of a converged warp, with one outcome for the warp
-__device__ __forceinline__ bool wait_bar_warp(uint64_t* bar, uint32_t parity, Ctrl* ctrl, int* status) {
-    const bool ok = wait_bar(bar, parity, ctrl, status);
-    return __all_sync(0xffffffffu, ok);
-}
-
-__device__ __forceinline__ void unit_coords(const TcParams& p, int u, int& mt, int& nt, int& sp) {
-    nt = u % p.tiles_n;
-    const int r = u / p.tiles_n;
-    mt = r % p.tiles_m;
-    sp = r / p.tiles_m;
-}
-
-// columns of column tile nt that the products cover: the whole tile, or what is left of the matrix rounded up
-__device__ __forceinline__ int tile_cols(const TcParams& p, int nt) {
-    const int left = (int)p.d.N - nt * p.bn;
-    return left >= p.bn ? p.bn : (left + p.n_gran - 1) / p.n_gran * p.n_gran;
-}
-
-__device__ __forceinline__ void unit_k_range(const TcParams& p, int sp, int64_t& kbeg, int& nkb, int& tail_steps) {
-    kbeg = (p.d.epi == EPI_PARTIAL) ? (int64_t)sp * p.d.k_per_split : 0;
-    int64_t kend = (p.d.epi == EPI_PARTIAL) ? kbeg + p.d.k_per_split : p.d.K;
-    if (kend > p.d.K) kend = p.d.K;
-    const int64_t len = kend - kbeg;
-    nkb = (int)((len + BK - 1) / BK);
-    const int rem = (int)(len - (int64_t)(nkb - 1) * BK);      // 1..BK elements in the last block
-    tail_steps = (rem + UMMA_K - 1) / UMMA_K;
-}
 
 // Sum over the 32 lanes of a warp of each of 32 per-lane values: lane l ends up with the total of v[l].
 // A butterfly of five exchange steps, so the order of the additions is fixed.
@@ -243,6 +197,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_init(smem_u32(&ctrl->reg_free[a]), NUM_EPI_WARPS + (CG == 2 ? 1 : 0));
         }
         ctrl->abort = 0;
+        ctrl->wait_limit = p.wait_limit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -265,7 +220,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         bool ok = true;
         for (int u = first_unit; u < p.units && ok; u += unit_step) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-            int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+            int64_t kbeg; int nkb, tail; unit_k_range<BK, UMMA_K>(p, sp, kbeg, nkb, tail);
             // this CTA's rows of A and its share of the tile's columns of B
             const int b_cols = tile_cols(p, nt) / CG;
             const int m0 = (mt * CG + rank) * BM, n0 = nt * p.bn + rank * b_cols;
@@ -333,7 +288,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         bool ok = get_a || get_b || get_a_lo || get_b_lo;
         for (int u = first_unit; u < p.units && ok; u += unit_step) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-            int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+            int64_t kbeg; int nkb, tail; unit_k_range<BK, UMMA_K>(p, sp, kbeg, nkb, tail);
             // this CTA's rows of A and its share of the tile's columns of B
             const int b_cols = tile_cols(p, nt) / CG;
             const int m0 = (mt * CG + rank) * BM, n0 = nt * p.bn + rank * b_cols;
@@ -410,7 +365,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             bool ok = true;
             for (int u = first_unit; u < p.units && ok; u += unit_step, ++tile_i) {
                 int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-                int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+                int64_t kbeg; int nkb, tail; unit_k_range<BK, UMMA_K>(p, sp, kbeg, nkb, tail);
                 const uint32_t idesc = idesc0 | ((uint32_t)(tile_cols(p, nt) >> 3) << 17);
                 const uint32_t total_reg = tile_i & 1;
                 uint32_t reg = total_reg, d_tmem = 0;
@@ -470,7 +425,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             bool ok = true;
             for (int u = first_unit; u < p.units && ok; u += unit_step) {
                 int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-                int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+                int64_t kbeg; int nkb, tail; unit_k_range<BK, UMMA_K>(p, sp, kbeg, nkb, tail);
                 for (int kb = 0; kb < nkb; ++kb) {
                     const int s = rp.stage;
                     uint64_t* bar = SPLIT ? &ctrl->ready[s] : &ctrl->full[s];
@@ -496,7 +451,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         bool ok = true;
         for (int u = first_unit; u < p.units && ok; u += unit_step, ++tile_i) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-            int64_t kbeg_; int nkb_, tail_; unit_k_range(p, sp, kbeg_, nkb_, tail_);
+            int64_t kbeg_; int nkb_, tail_; unit_k_range<BK, UMMA_K>(p, sp, kbeg_, nkb_, tail_);
             const int n_chunks = (nkb_ + p.chunk_blocks - 1) / p.chunk_blocks;
             const uint32_t acc = tile_i & 1, oth = acc ^ 1;
             const int n0 = nt * p.bn;
@@ -681,14 +636,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             tma_store_3d(map, smem_u32(blk), c0, r0w, EPI == EPI_PARTIAL ? sp : 0);
                             bulk_commit();
                         }
-                    } else if (rv) {
-                        float* dst = direct_base + r * ld + c0;
-                        if ((EPI == EPI_PARTIAL || c_vec) && full) {
+                    } else {
+                        // rows that TMA cannot address (a leading dimension that is not a multiple of four, a base that is
+                        // not 16-byte aligned): the block goes through the same staging block, and the warp then writes
+                        // it row by row, one 128-byte run per instruction
+                        uint8_t* blk = stg + (stg_i & 1) * EPI_STAGE_BYTES;
+                        ++stg_i;
+                        __syncwarp();
+                        float4* rowp = reinterpret_cast<float4*>(blk + lane * 128);
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(w[j], w[j + 1], w[j + 2], w[j + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = w[j];
+                        for (int j = 0; j < 8; ++j)
+                            rowp[j ^ (lane & 7)] = make_float4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                        __syncwarp();
+                        const int rows_here = min(32, (int)(d.M - r0w));
+                        if (lane < nvalid) {
+                            float* dst = direct_base + (int64_t)r0w * ld + c0 + lane;
+                            for (int rr = 0; rr < rows_here; ++rr) {
+                                const float* src = reinterpret_cast<const float*>(blk + rr * 128 + ((((lane >> 2) ^ (rr & 7)) << 4) | ((lane & 3) << 2)));
+                                dst[(int64_t)rr * ld] = *src;
+                            }
                         }
                     }
                 };
@@ -760,7 +726,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         bool ok = true;
         for (int u = first_unit; u < p.units && ok; u += unit_step) {
             int mt, nt, sp; unit_coords(p, u, mt, nt, sp);
-            int64_t kbeg; int nkb, tail; unit_k_range(p, sp, kbeg, nkb, tail);
+            int64_t kbeg; int nkb, tail; unit_k_range<BK, UMMA_K>(p, sp, kbeg, nkb, tail);
             const int m0 = (mt * CG + rank) * BM;
             const int b_cols = tile_cols(p, nt) / CG;
             // K-major logits (the pattern is the row): statistics of this thread's rows, once per tile
@@ -882,6 +848,31 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 }
 
+// One CTA, one warp: allocates tensor memory as the product kernels do, then waits (bounded) on a barrier that
+// nothing arrives on.  The wait gives up after `limit` cycles, records DEV_TIMEOUT, and the CTA leaves the way the
+// product kernels leave after an abort: tensor memory freed, nothing pending.
+__global__ void __launch_bounds__(32, 1) wait_probe_kernel(int* status, unsigned long long limit) {
+    __shared__ Ctrl ctrl_s;
+    Ctrl* ctrl = &ctrl_s;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&ctrl->full[0]), 1);
+        ctrl->abort = 0;
+        ctrl->wait_limit = limit;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    tmem_alloc<1>(smem_u32(&ctrl->tmem_base), 32);
+    tmem_relinquish<1>();
+    tc_fence_before();
+    __syncwarp();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+    (void)wait_bar_warp(&ctrl->full[0], 0, ctrl, status);      // phase 0 never completes
+    __syncwarp();
+    tc_fence_before();
+    tmem_dealloc<1>(tmem_base, 32);
+}
+
 // ------------------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -935,19 +926,19 @@ bool operand_ok(const float* base, int64_t s_major, int64_t s_minor_is_one_other
     return (((uintptr_t)base) & 15) == 0 && (s_major & 3) == 0 && s_major >= 4 && s_major < ((int64_t)1 << 38);
 }
 
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    }
-    return n;
-}
+int sm_count() { return sm_count_of_current_device(NUM_SMS); }
 
 int* status_ptr() {
-    static int* ptr = nullptr;
-    if (!ptr) { void* p = nullptr; if (cudaGetSymbolAddress(&p, g_dev_status) == cudaSuccess) ptr = (int*)p; }
+    static std::atomic<int*> cached[MAX_DEVICE_SLOTS];
+    const int slot = current_device_slot();
+    if (slot < 0) return nullptr;
+    int* ptr = cached[slot].load(std::memory_order_acquire);
+    if (!ptr) {
+        void* q = nullptr;
+        if (cudaGetSymbolAddress(&q, g_dev_status) != cudaSuccess) return nullptr;
+        ptr = (int*)q;
+        cached[slot].store(ptr, std::memory_order_release);
+    }
     return ptr;
 }
 
@@ -955,12 +946,8 @@ struct Maps { CUtensorMap a, b, a_lo, b_lo, c, c_lo; };
 
 template <int EPI, int CG, bool MULTI, bool THREE_X>
 ulsnn_status_t launch(const Maps& m, const TcParams& p, int smem_bytes, int grid, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<EPI, CG, MULTI, THREE_X>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) != cudaSuccess)
-            return ULSNN_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<uint64_t> configured{0};
+    if (!allow_dynamic_smem(tc_gemm_kernel<EPI, CG, MULTI, THREE_X>, SMEM_BUDGET, configured)) return ULSNN_ERR_CUDA;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
     cfg.blockDim = dim3(threads_of(MULTI), 1, 1);
@@ -1007,6 +994,8 @@ int tc_tile_n(const GemmDesc& d) {
     if (bn > BN_MAX) bn = BN_MAX;
     return (int)bn;
 }
+
+bool tc_operand_addressable(const float* base, int64_t ld) { return encode_fn() != nullptr && operand_ok(base, ld, 0); }
 
 bool tc_gemm_supported(const GemmDesc& d) {
     if (d.M <= 0 || d.N <= 0 || d.K <= 0) return false;
@@ -1059,6 +1048,7 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
     }
     p.status = status_ptr();
     if (!p.status) return ULSNN_ERR_CUDA;
+    p.wait_limit = DEFAULT_WAIT_LIMIT_CYCLES;
 
     Maps m;
     memset(&m, 0, sizeof(m));
@@ -1100,6 +1090,14 @@ ulsnn_status_t tc_gemm_launch(const GemmDesc& d, bool three_x, cudaStream_t stre
 }
 
 int* device_status_word() { return status_ptr(); }
+
+ulsnn_status_t tc_wait_probe_launch(unsigned long long limit_cycles, cudaStream_t stream) {
+    int* status = status_ptr();
+    if (!status) return ULSNN_ERR_CUDA;
+    wait_probe_kernel<<<1, 32, 0, stream>>>(status, limit_cycles);
+    count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
 
 ulsnn_status_t device_status_fetch_and_clear(cudaStream_t stream, int* word) {
     if (cudaStreamSynchronize(stream) != cudaSuccess) return ULSNN_ERR_CUDA;

@@ -4,6 +4,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <atomic>
+#include "common.cuh"
 
 namespace ulsnn {
 namespace {
@@ -194,6 +196,97 @@ struct RingPos {
     int stage; uint32_t phase;
     __device__ __forceinline__ void advance(int stages) { if (++stage == stages) { stage = 0; phase ^= 1u; } }
 };
+
+// Default limit of a device-side wait, in SM clock cycles (~1.5 s at 2 GHz): a kernel parameter, so that a test can
+// make a wait run out within microseconds.
+constexpr unsigned long long DEFAULT_WAIT_LIMIT_CYCLES = 3000000000ull;
+
+// Bounded wait on an mbarrier of a CTA whose control block `ctrl` has the fields `abort` and `wait_limit`.  Returns
+// false (after raising the abort flag and recording DEV_TIMEOUT in the device status word) if the phase did not
+// complete within the limit, or if another thread of the CTA has given up already.
+template <class CtrlT>
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, CtrlT* ctrl, int* status) {
+    const uint32_t b = smem_u32(bar);
+    if (mbar_try_wait(b, parity)) return true;
+    const unsigned long long t0 = clock64();
+    const unsigned long long limit = ctrl->wait_limit;
+    uint32_t spins = 0;
+    while (!mbar_try_wait(b, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (ctrl->abort) return false;
+            if ((unsigned long long)clock64() - t0 > limit) {
+                ctrl->abort = 1;
+                atomicExch(status, DEV_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+// wait_bar by all lanes of a converged warp, with one outcome for the warp
+template <class CtrlT>
+__device__ __forceinline__ bool wait_bar_warp(uint64_t* bar, uint32_t parity, CtrlT* ctrl, int* status) {
+    const bool ok = wait_bar(bar, parity, ctrl, status);
+    return __all_sync(0xffffffffu, ok);
+}
+
+// Work units of a persistent kernel: unit u = (column tile nt, row tile mt, split-K slice sp), nt fastest.  P has the
+// fields tiles_m, tiles_n, bn, n_gran and the product description d.
+template <class P>
+__device__ __forceinline__ void unit_coords(const P& p, int u, int& mt, int& nt, int& sp) {
+    nt = u % p.tiles_n;
+    const int r = u / p.tiles_n;
+    mt = r % p.tiles_m;
+    sp = r / p.tiles_m;
+}
+// columns of column tile nt that the products cover: the whole tile, or what is left of the matrix rounded up
+template <class P>
+__device__ __forceinline__ int tile_cols(const P& p, int nt) {
+    const int left = (int)p.d.N - nt * p.bn;
+    return left >= p.bn ? p.bn : (left + p.n_gran - 1) / p.n_gran * p.n_gran;
+}
+// k range of slice sp in blocks of BLOCK_K elements; tail_steps = product instructions (STEP_K elements each) of the last block
+template <int BLOCK_K, int STEP_K, class P>
+__device__ __forceinline__ void unit_k_range(const P& p, int sp, int64_t& kbeg, int& nkb, int& tail_steps) {
+    kbeg = (p.d.epi == EPI_PARTIAL) ? (int64_t)sp * p.d.k_per_split : 0;
+    int64_t kend = (p.d.epi == EPI_PARTIAL) ? kbeg + p.d.k_per_split : p.d.K;
+    if (kend > p.d.K) kend = p.d.K;
+    const int64_t len = kend - kbeg;
+    nkb = (int)((len + BLOCK_K - 1) / BLOCK_K);
+    const int rem = (int)(len - (int64_t)(nkb - 1) * BLOCK_K);      // 1..BLOCK_K elements in the last block
+    tail_steps = (rem + STEP_K - 1) / STEP_K;
+}
+
+// ------------------------------------------------------------------------------------------ per-device host state
+// One process may drive several GPUs, so whatever the host remembers about "the device" is kept per device ordinal.
+inline int current_device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    return device_cache_slot(dev);
+}
+inline int sm_count_of_current_device(int fallback) {
+    static std::atomic<int> cached[MAX_DEVICE_SLOTS];
+    const int slot = current_device_slot();
+    if (slot < 0) return fallback;
+    int n = cached[slot].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, slot) != cudaSuccess || n <= 0) n = fallback;
+        cached[slot].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) applies to the current device only: once per kernel and device.
+// `done` is the kernel's own bit mask over the device slots.
+template <class Kernel>
+inline bool allow_dynamic_smem(Kernel kernel, int bytes, std::atomic<uint64_t>& done) {
+    const int slot = current_device_slot();
+    if (slot < 0) return false;
+    const uint64_t bit = 1ull << slot;
+    if (done.load(std::memory_order_acquire) & bit) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    done.fetch_or(bit, std::memory_order_release);
+    return true;
+}
 
 }  // namespace
 }  // namespace ulsnn

@@ -156,3 +156,24 @@ def test_sixteen_bit_mode_workspaces():
     assert 65536 * 3208 * 2 < half < 0.7 * full
     with pytest.raises(ul.UlsnnError):
         ul.mlp_workspace_bytes([400, 480, 3203], 4, 65536)
+
+
+def test_per_device_tables_key_on_the_device_ordinal():
+    # every per-device cache of the library (architecture check, SM count, status-word address, kernel attributes,
+    # scratch buffers) is indexed by this slot: distinct devices get distinct slots, ordinals outside the table none
+    slots = [ul.device_cache_slot(d) for d in range(64)]
+    assert slots == list(range(64))
+    assert ul.device_cache_slot(-1) == -1 and ul.device_cache_slot(64) == -1 and ul.device_cache_slot(1 << 20) == -1
+
+
+def test_workspace_query_for_given_operands_is_host_only():
+    # no device: no operand is addressable by TMA and no tensor-core route exists, so the query equals the plain one;
+    # bad arguments are refused
+    for math in (ul.MATH_3XTF32, ul.MATH_TF32, ul.MATH_FP32_SIMT):
+        got = ul.sgemm_workspace_bytes_for("T", "N", 96, 200, 20000, 256, 96, 512, 200, math)
+        assert got >= 0
+    out = ctypes.c_size_t(0)
+    lib = ul.lib()
+    assert lib.ulsnn_sgemm_workspace_bytes_for(b"N", b"N", 4, 4, 4, None, 3, None, 4, 0, ctypes.byref(out)) == ul.ERR_INVALID_ARG
+    assert lib.ulsnn_sgemm_workspace_bytes_for(b"N", b"N", 4, 4, 4, None, 4, None, 4, 0, None) == ul.ERR_INVALID_ARG
+    assert lib.ulsnn_sgemm_workspace_bytes_for(b"N", b"N", 4, 4, 4, None, 4, None, 4, 9, ctypes.byref(out)) == ul.ERR_INVALID_ARG

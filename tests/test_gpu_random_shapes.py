@@ -8,7 +8,7 @@ import torch
 import oracle
 import synth_inputs as si
 from paper_1911_05181_b200 import binding as ul
-from helpers import TOL, GpuNet, dev, gpu_sgemm
+from helpers import TOL, GpuNet, dev, gpu_sgemm, tolerance_at
 
 pytestmark = pytest.mark.gpu
 
@@ -37,18 +37,16 @@ def test_random_sgemm_shapes(seed):
             if beta == 0.0:
                 C1[:, :N] = np.nan
             got = gpu_sgemm(ta, tb, M, N, K, alpha, A, lda, B, ldb, beta, C1, ldc, math)
-            # beta*C can cancel against alpha*AB: the low-precision modes get three times their tolerance
-            tol = TOL[math] * (1 if math in (ul.MATH_3XTF32, ul.MATH_FP32_SIMT) else 3)
-            assert oracle.rel_l2(got[:, :N], want) <= tol, (ta, tb, M, N, K, pad, alpha, beta, math)
+            assert oracle.rel_l2(got[:, :N], want) <= TOL[math], (ta, tb, M, N, K, pad, alpha, beta, math)
             if pad:
                 assert np.array_equal(got[:, N:], C[:, N:])
 
 
 def test_random_networks_both_heads():
     rng = np.random.default_rng(3)
-    for it in range(12):
+    for it in range(16):
         L = int(rng.integers(1, 4))
-        sizes = [int(rng.choice([8, 20, 33, 64, 100, 129, 256, 400])) for _ in range(L + 1)]
+        sizes = [int(rng.choice([3, 8, 20, 33, 64, 100, 129, 256, 400])) for _ in range(L + 1)]
         n = int(rng.choice([1, 5, 64, 127, 128, 129, 300, 1000, 2500]))
         seed = 500 + it
         Ws, bs = si.mlp_params(seed, sizes)
@@ -57,19 +55,20 @@ def test_random_networks_both_heads():
         T = si.mlp_targets(seed, sizes, n, 0, False)
         want = oracle.mlp_gradient(Ws, bs, X, y)
         want_sse = oracle.mlp_sse_gradient(Ws, bs, X, T)
+        # Every tensor is compared at the stated tolerance times max(1, its condition number / that of the benchmark
+        # network's worst tensor): layers of a few units make gradients whose relative sensitivity to perturbations
+        # of the inputs is several times the benchmark's, and no evaluation in finite precision can be held to more
+        cond = oracle.gradient_condition(Ws, bs, X, labels=y)
+        cond_sse = oracle.gradient_condition(Ws, bs, X, T=T)
         for math in MATHS:
             g = GpuNet(sizes, math, n); g.set_params(Ws, bs)
             got = g.gradient(X, y)
             g.net.gradient_sse(g.W, g.b, dev(X), sizes[0], dev(T), sizes[-1], n, False, g.dW, g.db, g.loss)
             torch.cuda.synchronize()
             got_sse = (float(g.loss.item()), [t.cpu().numpy() for t in g.dW], [t.cpu().numpy() for t in g.db])
-            # twice the tolerance of the benchmark networks: gradient tensors of a few elements are sums of thousands
-            # of terms that nearly cancel, so their relative error is larger (with 3-unit layers, which are left out
-            # here, 1.007e-5 was seen in 3xTF32 mode and 1.1e-2 in TF32 mode)
-            tol = 2 * TOL[math]
-            for a, b in ((got, want), (got_sse, want_sse)):
-                assert abs(a[0] - b[0]) <= tol * abs(b[0]), (sizes, n, math)
-                for u, v in zip(a[1] + a[2], b[1] + b[2]):
-                    assert oracle.rel_l2(u, v) <= tol, (sizes, n, math)
+            for head, a, b, c in (("softmax", got, want, cond), ("sse", got_sse, want_sse, cond_sse)):
+                assert abs(a[0] - b[0]) <= TOL[math] * abs(b[0]), (sizes, n, math, head)
+                for u, v, k in zip(a[1] + a[2], b[1] + b[2], c[0] + c[1]):
+                    assert oracle.rel_l2(u, v) <= tolerance_at(math, k, head), (sizes, n, math, head, k)
             assert g.net.last_device_status() == ul.OK
             g.net.close()

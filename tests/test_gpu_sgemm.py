@@ -109,3 +109,42 @@ def test_paper_shapes_sampled(math, shape):
     want = np.array([oracle.sgemm_entry(ta, tb, K, 1.0, A, lda, B, ldb, 0.0, None, 0, int(i), int(j)) for i, j in zip(ii, jj)])
     err = oracle.rel_l2(got[ii, jj], want)
     assert err <= TOL[math], err
+
+
+@pytest.mark.parametrize("math", [ul.MATH_3XTF32, ul.MATH_TF32])
+def test_operands_tma_cannot_address_are_rebuffered_onto_the_tensor_cores(math):
+    """Packed rows of 3203 floats (the class count of the paper's network is prime) and a base pointer that is not
+    16-byte aligned: with the workspace ulsnn_sgemm_workspace_bytes_for asks for, the product runs on the tensor-core
+    engine after a copy with padded rows (Section 3.3's re-buffering); with less, on the FFMA kernel.  Both are right."""
+    for ta, tb, M, N, K, off in (("N", "N", 700, 3203, 480, 0), ("T", "N", 480, 3203, 2100, 0), ("N", "T", 300, 130, 203, 1),
+                                 ("T", "T", 129, 65, 77, 3)):
+        ra, ca = (K, M) if ta == "T" else (M, K)
+        rb, cb = (N, K) if tb == "T" else (K, N)
+        A, B, C = si.gemm_operands(31, ra, ca, rb, cb, M, N)
+        want = oracle.sgemm(ta, tb, M, N, K, 1.0, A, ca, B, cb, 0.5, C.copy(), N)
+        # device copies shifted by `off` floats: bases that are 4-byte but not 16-byte aligned
+        bufA = torch.empty(A.size + 8, device="cuda"); bufB = torch.empty(B.size + 8, device="cuda")
+        dA = bufA[off:off + A.size].view(ra, ca); dB = bufB[off:off + B.size].view(rb, cb)
+        dA.copy_(torch.from_numpy(A)); dB.copy_(torch.from_numpy(B))
+        plain = ul.sgemm_workspace_bytes(ta, tb, M, N, K, math)
+        need = ul.sgemm_workspace_bytes_for(ta, tb, M, N, K, dA, ca, dB, cb, math)
+        assert need > plain
+        for nbytes, tc_expected in ((need, True), (plain, False)):
+            ws = torch.empty(max(nbytes, 1) + 256, dtype=torch.uint8, device="cuda")
+            wp = (ws.data_ptr() + 255) // 256 * 256
+            dC = dev(C)
+            c0 = ul.launch_counts()
+            ul.sgemm_ex(ta, tb, M, N, K, 1.0, dA, ca, dB, cb, 0.5, dC, N, math, wp if nbytes else None, nbytes)
+            torch.cuda.synchronize()
+            c1 = ul.launch_counts()
+            assert (c1["tc_gemm"] > c0["tc_gemm"]) == tc_expected and (c1["simt_gemm"] > c0["simt_gemm"]) == (not tc_expected)
+            tol = TOL[math] if tc_expected else TOL[ul.MATH_FP32_SIMT]
+            assert oracle.rel_l2(dC.cpu().numpy(), want) <= tol, (ta, tb, M, N, K, off, nbytes)
+        # the allocating entry point takes the re-buffered route by itself
+        if math == ul.MATH_3XTF32:
+            dC = dev(C)
+            c0 = ul.launch_counts()
+            ul.sgemm(ta, tb, M, N, K, 1.0, dA, ca, dB, cb, 0.5, dC, N)
+            torch.cuda.synchronize()
+            assert ul.launch_counts()["tc_gemm"] > c0["tc_gemm"]
+            assert oracle.rel_l2(dC.cpu().numpy(), want) <= TOL[math]

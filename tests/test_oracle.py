@@ -288,3 +288,88 @@ def test_untrained_classifier_loss_is_near_ln_classes():
     X, y = si.mlp_batch(0, sizes, 512)
     loss = oracle.mlp_forward_loss(Ws, bs, X, y)
     assert 512 * math.log(64) < loss < 1.2 * 512 * math.log(64)
+
+
+# ----------------------------------------------------------------------------- magnitude sums and condition numbers
+
+@pytest.mark.parametrize("transA", ["N", "T"])
+@pytest.mark.parametrize("transB", ["N", "T"])
+def test_sgemm_abs_small_integers_exact(transA, transB):
+    # |alpha| sum_k |a||b| + |beta||c| against a pure-Python loop; equal to the product itself when nothing is negative
+    rng = np.random.default_rng(11)
+    M, N, K = 4, 3, 5
+    ra, ca = (K, M) if transA == "T" else (M, K)
+    rb, cb = (N, K) if transB == "T" else (K, N)
+    A = rng.integers(-4, 5, (ra, ca)).astype(np.float32); B = rng.integers(-4, 5, (rb, cb)).astype(np.float32)
+    C = rng.integers(-4, 5, (M, N)).astype(np.float32)
+    got = oracle.sgemm_abs(transA, transB, M, N, K, -3.0, A, ca, B, cb, -2.0, C, N)
+    want = _brute(transA, transB, M, N, K, 3.0, np.abs(A).tolist(), np.abs(B).tolist(), 2.0, np.abs(C).tolist())
+    assert np.array_equal(got, np.asarray(want, dtype=np.float64))
+    pos = oracle.sgemm(transA, transB, M, N, K, 3.0, np.abs(A), ca, np.abs(B), cb, 2.0, np.abs(C), N)
+    assert np.array_equal(got, pos)
+
+
+def test_gradient_magnitudes_hand_worked_2_1_2():
+    # the hand-worked network: softmax (2/3, 1/3), label 0 -> output magnitudes (2/3 + 1, 1/3), h = 1/2,
+    # hidden magnitude (1 - h^2) * (|2 ln 2| * 5/3 + 0 * 1/3)
+    with open(os.path.join(GOLD, "hand_net_2_1_2.json")) as f:
+        g = json.load(f)
+    W1 = np.asarray(_ev(g["W1"]), np.float32); W2 = np.asarray(_ev(g["W2"]), np.float32)
+    b1 = np.asarray(_ev(g["b1"]), np.float32); b2 = np.asarray(_ev(g["b2"]), np.float32)
+    X = np.asarray([_ev(g["x"])], np.float32)
+    aW, ab = oracle.mlp_gradient_abs([W1, W2], [b1, b2], X, labels=np.asarray([0], np.int32))
+    m1 = 0.75 * (2 * math.log(2) * 5 / 3)
+    # fp32 storage of ln(3)/2 and 2 ln 2 moves the values by ~1e-8 relative
+    assert np.allclose(ab[1], [5 / 3, 1 / 3], rtol=1e-6) and np.allclose(aW[1], [[5 / 6], [1 / 6]], rtol=1e-6)
+    assert np.allclose(ab[0], [m1], rtol=1e-6) and np.allclose(aW[0], [[m1, 0.0]], rtol=1e-6)
+
+
+@pytest.mark.parametrize("head", ["softmax", "sse"])
+def test_gradient_magnitudes_bound_the_gradient(head):
+    sizes, n = [6, 5, 4, 3], 40
+    Ws, bs = si.mlp_params(21, sizes)
+    bs = [(0.3 * si.uniform_pm1(21, 11 + i, b.size)).astype(np.float32) for i, b in enumerate(bs)]
+    X, y = si.mlp_batch(21, sizes, n)
+    T = si.mlp_targets(21, sizes, n)
+    if head == "softmax":
+        _, gW, gb = oracle.mlp_gradient(Ws, bs, X, y); aW, ab = oracle.mlp_gradient_abs(Ws, bs, X, labels=y)
+    else:
+        _, gW, gb = oracle.mlp_sse_gradient(Ws, bs, X, T); aW, ab = oracle.mlp_gradient_abs(Ws, bs, X, T=T)
+    for g_, a_ in zip(gW + gb, aW + ab):
+        assert (a_ >= np.abs(g_) * (1 - 1e-12)).all() and (a_ > 0).all()
+    # one pattern, one weight matrix, squared-error head: every entry is a single product, so magnitude = |gradient|
+    _, g1W, g1b = oracle.mlp_sse_gradient(Ws[:1], bs[:1], X[:1], T[:1, :sizes[1]])
+    a1W, a1b = oracle.mlp_gradient_abs(Ws[:1], bs[:1], X[:1], T=T[:1, :sizes[1]])
+    assert np.allclose(a1W[0], np.abs(g1W[0]), rtol=1e-13) and np.allclose(a1b[0], np.abs(g1b[0]), rtol=1e-13)
+
+
+def test_gradient_condition_of_a_gradient_linear_in_the_pattern():
+    # all-zero parameters, one pattern: dW = (1/n_o - onehot) x^T does not depend on W and is linear in x, so its
+    # relative change under x -> x~ is ||x~ - x|| / ||x|| exactly; db does not depend on x at all
+    sizes = [7, 4]
+    W = [np.zeros((4, 7), np.float32)]; b = [np.zeros(4, np.float32)]
+    X = (0.25 + si.uniform01(5, si.TID_X, 7)).reshape(1, 7).astype(np.float32)
+    y = np.asarray([2], np.int32)
+    eps, seeds = 2.0 ** -14, (12345, 12346)
+    cW, cb = oracle.gradient_condition(W, b, X, labels=y, eps=eps, seeds=seeds)
+    want = 0.0
+    for s in seeds:
+        _, _, Xp, _ = oracle.perturb_inputs(W, b, X, None, eps, s)
+        want = max(want, np.linalg.norm((Xp.astype(np.float64) - X).ravel()) / np.linalg.norm(X.astype(np.float64).ravel()))
+    assert abs(cW[0] - want / (eps / math.sqrt(3))) < 1e-6 * cW[0]
+    assert 0.3 < cW[0] < 3.0 and cb[0] == 0.0
+
+
+def test_condition_reference_of_the_benchmark_network_is_stored():
+    with open(os.path.join(GOLD, "cond_ref.json")) as f:
+        ref = json.load(f)
+    vals = ref["softmax"]["dW"] + ref["softmax"]["db"] + ref["sse"]["dW"] + ref["sse"]["db"]
+    assert ref["cond_ref"] == max(vals) and all(0.5 < v < 3.0 for v in vals)
+    # a 1/16 sample of the stored configuration reproduces the weight-gradient values, which set the maximum, to
+    # 15 % (they do not depend on the batch; the top bias gradient's does: its label counts are exact)
+    sizes = [400, 480, 3203]
+    Ws, bs = si.mlp_params(2, sizes)
+    X, y = si.mlp_batch(2, sizes, 512)
+    cW, cb = oracle.gradient_condition(Ws, bs, X, labels=y, seeds=(12345,))
+    for got, want in zip(cW + cb[:1], ref["softmax"]["dW"] + ref["softmax"]["db"][:1]):
+        assert abs(got - want) < 0.15 * want

@@ -26,11 +26,12 @@ def _operands(ta, tb, M, N, K, seed):
 
 
 def _ex(ta, tb, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, math):
-    nbytes = ul.sgemm_workspace_bytes(ta, tb, M, N, K, math)
+    dA, dB = dev(A), dev(B)
+    nbytes = ul.sgemm_workspace_bytes_for(ta, tb, M, N, K, dA, lda, dB, ldb, math)
     ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
     wp = (ws.data_ptr() + 255) // 256 * 256
     dC = dev(C)
-    ul.sgemm_ex(ta, tb, M, N, K, alpha, dev(A), lda, dev(B), ldb, beta, dC, ldc, math, wp if nbytes else None, nbytes)
+    ul.sgemm_ex(ta, tb, M, N, K, alpha, dA, lda, dB, ldb, beta, dC, ldc, math, wp if nbytes else None, nbytes)
     torch.cuda.synchronize()
     return dC.cpu().numpy(), nbytes
 
@@ -76,3 +77,35 @@ def test_products_without_split_and_oversized_products():
     assert st == ul.ERR_TOO_LARGE
     torch.cuda.synchronize()
     assert bool((c == 7.0).all())
+
+
+def test_sixteen_bit_mode_padded_rows_and_degenerate_products():
+    """The branches the two-call test leaves out.  The 16-bit mode keeps its bfloat16 operand copies in the array as well, so
+    only small products fit; operands whose rows TMA cannot address are re-buffered in the array when copies and partials
+    fit; K == 0 and alpha == 0 touch neither operands nor array.  Each is held bit for bit against the workspace entry point."""
+    # 16-bit mode, accepted: copies of A (128 x 2048) and B (2048 x 96) plus partials are well below 8 MiB
+    for _ in range(2):
+        A, lda, B, ldb, C, ldc = _operands("N", "N", 128, 96, 2048, 11)
+        want, nbytes = _ex("N", "N", 128, 96, 2048, 1.0, A, lda, B, ldb, 0.5, C, ldc, ul.MATH_BF16)
+        assert 0 < nbytes <= ul.sgemm_noalloc_max_scratch_bytes()
+        got = _noalloc("N", "N", 128, 96, 2048, 1.0, A, lda, B, ldb, 0.5, C, ldc, ul.MATH_BF16)
+        assert np.array_equal(got, want)
+        assert oracle.rel_l2(got, oracle.sgemm("N", "N", 128, 96, 2048, 1.0, A, lda, B, ldb, 0.5, C, ldc)) <= TOL[ul.MATH_BF16]
+    # 16-bit mode, rejected: the copies alone (2 x 2048 x 2048 bfloat16 = 16 MiB) exceed the array
+    z = torch.zeros(2048, 2048, device="cuda"); c = torch.full((2048, 2048), 3.0, device="cuda")
+    assert ul.sgemm_noalloc("N", "N", 2048, 2048, 2048, 1.0, z, 2048, z, 2048, 0.0, c, 2048, ul.MATH_BF16, check=False) == ul.ERR_TOO_LARGE
+    torch.cuda.synchronize()
+    assert bool((c == 3.0).all())
+    # rows of 130 floats (not a multiple of 4): copies and partials fit, both entry points take the re-buffered route
+    for math in (ul.MATH_3XTF32, ul.MATH_TF32):
+        A, lda, B, ldb, C, ldc = _operands("T", "N", 130, 66, 9000, 12)
+        want, nbytes = _ex("T", "N", 130, 66, 9000, 1.5, A, lda, B, ldb, 1.0, C, ldc, math)
+        assert 0 < nbytes <= ul.sgemm_noalloc_max_scratch_bytes()
+        got = _noalloc("T", "N", 130, 66, 9000, 1.5, A, lda, B, ldb, 1.0, C, ldc, math)
+        assert np.array_equal(got, want)
+        assert oracle.rel_l2(got, oracle.sgemm("T", "N", 130, 66, 9000, 1.5, A, lda, B, ldb, 1.0, C, ldc)) <= TOL[math]
+    # K == 0 and alpha == 0: C = beta * C, operands never read (they hold NaN)
+    nan = np.full((8, 8), np.nan, np.float32); C = si.uniform_pm1(3, 9, 64).reshape(8, 8)
+    for math in (ul.MATH_3XTF32, ul.MATH_BF16):
+        assert np.array_equal(_noalloc("N", "N", 8, 8, 0, 1.0, nan, 8, nan, 8, 2.0, C.copy(), 8, math), 2.0 * C)
+        assert np.array_equal(_noalloc("N", "N", 8, 8, 8, 0.0, nan, 8, nan, 8, 1.0, C.copy(), 8, math), C)
