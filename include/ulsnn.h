@@ -197,6 +197,17 @@ ulsnn_status_t ulsnn_mlp_gradient_sse(ulsnn_mlp_t* handle, const float* const* W
                                       int accumulate, float* const* dW, float* const* db, double* loss_out,
                                       ulsnn_stream_t stream);
 /* Section 4.2: W := W - lr * dW, b := b - lr * db, in place, one fused multiply-add per element. */
+/*
+ * Training-set parallelism over several GPUs (Section 4.3: the patterns are partitioned, every worker evaluates its
+ * share, the per-worker gradients are summed).  events: host array of n_layers CUDA events (cudaEvent_t, created by
+ * the caller; entries may be NULL), or NULL to switch this off.  Every later ulsnn_mlp_gradient[_sse] on the handle
+ * records events[w] on its stream as soon as dW[w] and db[w] of that call are final: the top layer's come first, the
+ * first layer's last, so the exchange of a layer's gradient with the other GPUs can run on a second stream while the
+ * products of the layers below still compute (the reduce overlapped with computation, Section 5.2).  The events stay
+ * the caller's; the handle keeps the array's entries, not the array.
+ */
+ulsnn_status_t ulsnn_mlp_set_gradient_events(ulsnn_mlp_t* handle, void* const* events /* host */);
+
 ulsnn_status_t ulsnn_sgd_step(ulsnn_mlp_t* handle, float* const* W, float* const* b,
                               const float* const* dW, const float* const* db, float lr, ulsnn_stream_t stream);
 /*

@@ -34,6 +34,7 @@ EXPORTS = [
     "ulsnn_sgemm_noalloc", "ulsnn_sgemm_noalloc_max_scratch_bytes", "ulsnn_mlp_forward_sse", "ulsnn_mlp_gradient_sse",
     "ulsnn_vec_dot_workspace_bytes", "ulsnn_vec_dot", "ulsnn_vec_axpby",
     "ulsnn_sgemm_workspace_bytes_for", "ulsnn_debug_wait_timeout", "ulsnn_debug_device_cache_slot",
+    "ulsnn_mlp_set_gradient_events",
 ]
 
 
@@ -89,6 +90,7 @@ def lib():
         l.ulsnn_vec_axpby.argtypes = [i64, f32, vp, f32, vp, vp, vp]
         l.ulsnn_sgd_step.argtypes = [vp, pp, pp, pp, pp, f32, vp]
         l.ulsnn_last_device_status.argtypes = [vp, vp]
+        l.ulsnn_mlp_set_gradient_events.argtypes = [vp, pp]
         l.ulsnn_fill_uniform.argtypes = [vp, i64, u64, u64, u64, ctypes.c_int, vp]
         l.ulsnn_fill_labels.argtypes = [vp, i64, u64, u64, u64, i32, vp]
         l.ulsnn_launch_counts.argtypes = [ctypes.POINTER(i64)]
@@ -304,6 +306,14 @@ class Mlp:
         n = ctypes.c_int(cap); ms = (ctypes.c_float * cap)(); mnk = (ctypes.c_int64 * (3 * cap))()
         _check(lib().ulsnn_mlp_phase_times(self._h, ctypes.byref(n), ms, mnk), "ulsnn_mlp_phase_times")
         return [(ms[i], mnk[3 * i], mnk[3 * i + 1], mnk[3 * i + 2]) for i in range(n.value)]
+
+    def set_gradient_events(self, events):
+        """events: one torch.cuda.Event (already recorded once, so that it exists) or None per weight matrix, or None."""
+        if events is None:
+            _check(lib().ulsnn_mlp_set_gradient_events(self._h, None), "ulsnn_mlp_set_gradient_events")
+            return
+        arr = (ctypes.c_void_p * len(events))(*[(e.cuda_event if e is not None else None) for e in events])
+        _check(lib().ulsnn_mlp_set_gradient_events(self._h, arr), "ulsnn_mlp_set_gradient_events")
 
     def last_device_status(self, stream=None) -> int:
         return lib().ulsnn_last_device_status(self._h, _stream(stream))

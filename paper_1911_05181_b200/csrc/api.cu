@@ -457,6 +457,9 @@ struct ulsnn_mlp {
     __nv_bfloat16* Hb[MAX_LAYERS + 1]; int64_t ldhb[MAX_LAYERS + 1];
     __nv_bfloat16* Db[MAX_LAYERS + 1]; int64_t lddb[MAX_LAYERS + 1];
     __nv_bfloat16* Eb; int64_t ldeb;
+    // optional: events recorded when the gradient of a weight matrix (dW_w and db_w) is final
+    cudaEvent_t grad_done[MAX_LAYERS];
+    bool have_grad_events;
     // optional per-product timing
     bool timing;
     int n_phases;                       // products launched so far by the call in flight
@@ -623,6 +626,13 @@ ulsnn_status_t timed_gemm(ulsnn_mlp* h, const HalfGemmDesc& d, cudaStream_t stre
     return timed_product(h, d.M, d.N, d.K, stream, [&] { return hg_gemm_launch(d, stream); });
 }
 
+// dW_w and db_w of this call are final on the stream: tell whoever waits for them (the gradient exchange between
+// several GPUs starts on a layer's gradient while the products of the layers below still run)
+ulsnn_status_t mark_gradient_done(ulsnn_mlp* h, int w, cudaStream_t stream) {
+    if (!h->have_grad_events || !h->grad_done[w]) return ULSNN_OK;
+    return cuda_ok(cudaEventRecord(h->grad_done[w], stream));
+}
+
 // The forward products: hidden layers with bias + tanh fused, then the logits with their row statistics.
 // What the outputs are compared with: integer labels (softmax + cross-entropy) or, when T is not null, a dense
 // target matrix (the paper's tanh outputs with summed squared error, Eqs. 1 and 3).
@@ -763,6 +773,7 @@ ulsnn_status_t gradient_bf16(ulsnn_mlp* h, const float* const* W, const float* c
         if ((size_t)p.splits * (size_t)d.M * (size_t)d.ldp * sizeof(float) > h->partials_bytes) return ULSNN_ERR_WORKSPACE_TOO_SMALL;
         if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
         if ((st = launch_splitk_reduce(d.partials, p.splits, d.M, h->sizes[w], d.ldp, 1.f, beta, dW[w], h->sizes[w], db[w], stream)) != ULSNN_OK) return st;
+        if ((st = mark_gradient_done(h, w, stream)) != ULSNN_OK) return st;
     }
     return ULSNN_OK;
 }
@@ -805,6 +816,18 @@ extern "C" void ulsnn_mlp_destroy(ulsnn_mlp_t* handle) {
     if (!handle) return;
     for (cudaEvent_t e : handle->ev) if (e) cudaEventDestroy(e);
     delete handle;
+}
+
+extern "C" ulsnn_status_t ulsnn_mlp_set_gradient_events(ulsnn_mlp_t* h, void* const* events) {
+    if (!h) return ULSNN_ERR_INVALID_ARG;
+    h->have_grad_events = false;
+    for (int w = 0; w < MAX_LAYERS; ++w) h->grad_done[w] = nullptr;
+    if (!events) return ULSNN_OK;
+    for (int w = 0; w < h->L; ++w) {
+        h->grad_done[w] = (cudaEvent_t)events[w];
+        if (events[w]) h->have_grad_events = true;
+    }
+    return ULSNN_OK;
 }
 
 extern "C" ulsnn_status_t ulsnn_mlp_enable_timing(ulsnn_mlp_t* h, int on) {
@@ -933,6 +956,7 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
         if ((st = timed_gemm(h, d, stream)) != ULSNN_OK) return st;
         if ((st = launch_splitk_reduce(d.partials, p.splits, d.M, h->sizes[w], d.ldp, 1.f, beta, dW[w], h->sizes[w],
                                        w >= 1 ? db[w] : nullptr, stream)) != ULSNN_OK) return st;
+        if (w >= 1 && (st = mark_gradient_done(h, w, stream)) != ULSNN_OK) return st;
     }
     // bias gradient of the first layer: column sums of delta_1 (both engines use 128-row tiles)
     if (L >= 2) {
@@ -942,7 +966,8 @@ ulsnn_status_t gradient_call(ulsnn_mlp_t* h, const float* const* W, const float*
     } else {
         st = launch_delta_colsum(h->Z, h->ldz, h->chunk_tab, h->chunk_ld, labels, n, h->sizes[1], h->colsum_parts, accumulate, db[0], stream);
     }
-    return st;
+    if (st != ULSNN_OK) return st;
+    return mark_gradient_done(h, 0, stream);      // db_0 comes last
 }
 
 }  // namespace

@@ -65,7 +65,8 @@ constexpr int NUM_SMS = 148;               // B200; fixes the tile schedule (and
 constexpr int A_TILE_BYTES = BM * BK * 4;
 constexpr int SMEM_BUDGET = 227 * 1024;
 constexpr int EPI_STAGE_BYTES = 32 * 128;                        // one 32x32 fp32 block, 128B-swizzled
-constexpr int EPI_SCRATCH_BYTES = NUM_EPI_WARPS * 2 * EPI_STAGE_BYTES;   // two store-staging blocks per epilogue warp
+constexpr int EPI_BIAS_BYTES = BN_MAX * 4;                       // a tile's bias values, shared by the epilogue warps
+constexpr int EPI_SCRATCH_BYTES = NUM_EPI_WARPS * 2 * EPI_STAGE_BYTES + EPI_BIAS_BYTES;   // two store-staging blocks per epilogue warp + the bias copy
 constexpr int CTRL_BYTES = 1024;                                // barriers, TMEM base, abort flag
 
 struct TcParams {
@@ -99,6 +100,7 @@ struct Ctrl {
     uint64_t reg_free[2];           // the epilogue warps have read region r: it may be overwritten
     uint64_t relay_sink[MAX_STAGES];    // CTA 0: landing words of CTA 1's stage-ready signals
     uint64_t free_sink[2][NUM_EPI_WARPS];   // CTA 0: landing words of CTA 1's accumulator-free signals
+    uint64_t bias_full, bias_free;  // the tile's bias copy has been written / read by all epilogue warps
     uint32_t tmem_base;
     volatile int abort;
     unsigned long long wait_limit;
@@ -196,6 +198,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // CTA 1's epilogue warps will signal
             mbar_init(smem_u32(&ctrl->reg_free[a]), NUM_EPI_WARPS + (CG == 2 ? 1 : 0));
         }
+        mbar_init(smem_u32(&ctrl->bias_full), NUM_EPI_WARPS);
+        mbar_init(smem_u32(&ctrl->bias_free), NUM_EPI_WARPS);
         ctrl->abort = 0;
         ctrl->wait_limit = p.wait_limit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -441,9 +445,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int q = warp & 3;                         // TMEM lane quarter this warp may read
         const int ew = warp - 2;                        // 0..3, index of this warp among the epilogue warps
         uint8_t* stg = epi_scratch + ew * (2 * EPI_STAGE_BYTES);     // two 32x32 store-staging blocks of this warp
+        // The tile's bias values, one copy for the four epilogue warps (each writes a quarter): fetched from global
+        // memory block by block they cost a third of a block's time, and shared memory has 1 KB to spare, not 4.
+        float* bias_s = reinterpret_cast<float*>(epi_scratch + NUM_EPI_WARPS * (2 * EPI_STAGE_BYTES));
+        constexpr bool HAS_BIAS = EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS || EPI == EPI_TANH_SSE;
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
         const bool c_vec = ((((uintptr_t)d.C) & 15) == 0) && ((d.ldc & 3) == 0);
-        const bool bias_vec = (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS || EPI == EPI_TANH_SSE) && ((((uintptr_t)d.bias) & 15) == 0);
         const bool t_vec = (EPI == EPI_TANH_SSE) && ((((uintptr_t)d.T) & 15) == 0) && ((d.ldt & 3) == 0);
         const bool h_vec = (EPI == EPI_TANHP) && ((((uintptr_t)d.Hm) & 15) == 0) && ((((uintptr_t)d.Hm_lo) & 15) == 0) && ((d.ldh & 3) == 0);
         uint32_t tile_i = 0, stg_i = 0;
@@ -456,6 +463,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t acc = tile_i & 1, oth = acc ^ 1;
             const int n0 = nt * p.bn;
             const int chunks = (min(p.bn, (int)d.N - n0) + 31) >> 5;       // 32-column blocks of this tile inside the matrix
+            if (HAS_BIAS) {
+                // before the wait for the tile's products, so that the loads hide behind them; the copy may be
+                // overwritten once every epilogue warp is through with the previous tile
+                if (tile_i > 0 && !wait_bar(&ctrl->bias_free, (tile_i - 1) & 1, ctrl, p.status)) { ok = false; break; }
+                constexpr int PER_WARP = BN_MAX / NUM_EPI_WARPS;        // 64 values per warp
+#pragma unroll
+                for (int j = 0; j < PER_WARP / 32; ++j) {
+                    const int idx = ew * PER_WARP + j * 32 + lane;
+                    bias_s[idx] = n0 + idx < (int)d.N ? __ldg(d.bias + n0 + idx) : 0.f;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->bias_full));
+            }
             if (!wait_bar(&ctrl->reg_full[acc], reads[acc] & 1, ctrl, p.status)) { ok = false; break; }
             reads[acc]++;
             tc_fence_after();
@@ -479,6 +499,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (lane == 0) { if (CG == 2 && rank == 1) signal_rank0(smem_u32(&ctrl->free_sink[oth][ew]), smem_u32(&ctrl->reg_free[oth])); else mbar_arrive(smem_u32(&ctrl->reg_free[oth])); }
             }
             if (!ok) break;
+            if (HAS_BIAS && !wait_bar(&ctrl->bias_full, tile_i & 1, ctrl, p.status)) { ok = false; break; }
             const int r0w = (mt * CG + rank) * BM + q * 32;   // first row of this warp's 32-row block
             const int64_t r = (int64_t)r0w + lane;
             const bool rv = r < d.M;
@@ -522,15 +543,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int j = 0; j < 32; ++j) v[j] = d.alpha * v[j];
                     }
                 } else if (EPI == EPI_BIAS_TANH || EPI == EPI_LOGITS || EPI == EPI_TANH_SSE) {
-                    if (bias_vec && full) {
+                    {
+                        const float4* bs = reinterpret_cast<const float4*>(bias_s + c * 32);      // every lane reads the same words
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
-                            const float4 bb = __ldg(reinterpret_cast<const float4*>(d.bias + c0 + j));
+                            const float4 bb = bs[j >> 2];
                             v[j] += bb.x; v[j + 1] += bb.y; v[j + 2] += bb.z; v[j + 3] += bb.w;
                         }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) if (j < nvalid) v[j] += __ldg(d.bias + c0 + j);
                     }
                     if (EPI == EPI_BIAS_TANH) {
 #pragma unroll
@@ -683,6 +702,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // all TMEM reads of this accumulator stage are done: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
+            if (HAS_BIAS && lane == 0) mbar_arrive(smem_u32(&ctrl->bias_free));
             if (lane == 0) { if (CG == 2 && rank == 1) signal_rank0(smem_u32(&ctrl->free_sink[acc][ew]), smem_u32(&ctrl->reg_free[acc])); else mbar_arrive(smem_u32(&ctrl->reg_free[acc])); }
 
             if (EPI == EPI_TANH_SSE && rv) d.stats[r * d.stats_ld + nt] = make_float2(0.f, run_s);

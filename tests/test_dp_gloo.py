@@ -90,3 +90,64 @@ def test_single_rank_exchange_is_a_no_op():
     loss = torch.tensor([2.5], dtype=torch.float64)
     dp.GradientExchange(g, None).all_reduce(g, loss)
     assert all(torch.equal(a, b) for a, b in zip(g, before)) and loss.item() == 2.5
+
+
+# ---- fixed total number of patterns (the processor-scaling experiment of Section 6.3) and the exchange launched
+# ---- layer by layer while the rest of the gradient is still being computed (Section 5.2)
+
+TOTAL = 75          # not a multiple of the world size: the first rank gets one pattern more
+
+
+def _worker_strong(rank, world, port, out_dir, ordered, overlapped):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        Ws, bs = si.mlp_params(SEED, SIZES)
+        first, last = dp.split_range(TOTAL, world, rank)
+        X, y = si.mlp_batch(SEED, SIZES, last - first, offset=first)
+        loss, dW, db = oracle.mlp_gradient(Ws, bs, X, y)
+        grads = [torch.from_numpy(np.ascontiguousarray(g)) for g in dW + db]
+        loss_t = torch.tensor([loss], dtype=torch.float64)
+        L = len(SIZES) - 1
+        if overlapped:
+            ex = dp.GradientExchange(grads, dist, ordered=ordered, groups=dp.layer_groups(L))
+            for g in range(L - 1):           # the top layers' gradients leave early, the last group leaves in finish()
+                ex.start(g, grads)
+            ex.finish(grads, loss_t)
+        else:
+            ex = dp.GradientExchange(grads, dist, ordered=ordered)
+            ex.all_reduce(grads, loss_t)
+        np.savez(os.path.join(out_dir, "rank%d_%d.npz" % (rank, int(overlapped))), loss=loss_t.numpy(), first=first, last=last,
+                 *[g.numpy() for g in grads])
+    finally:
+        dist.destroy_process_group()
+
+
+def test_layer_groups_follow_the_order_in_which_gradients_become_final():
+    assert dp.layer_groups(2) == [[1, 3], [0, 2]]
+    assert dp.layer_groups(3) == [[2, 5], [1, 4], [0, 3]]
+    with pytest.raises(ValueError):
+        dp.GradientExchange([torch.zeros(2), torch.zeros(3)], None, groups=[[0]])
+
+
+@pytest.mark.parametrize("ordered", [False, True])
+def test_fixed_total_split_and_overlapped_exchange_give_the_serial_bits(tmp_path, ordered):
+    world = 2
+    for overlapped in (False, True):
+        mp.spawn(_worker_strong, args=(world, _free_port(), str(tmp_path), ordered, overlapped), nprocs=world, join=True)
+    Ws, bs = si.mlp_params(SEED, SIZES)
+    X, y = si.mlp_batch(SEED, SIZES, TOTAL)
+    loss, dW, db = oracle.mlp_gradient(Ws, bs, X, y)
+    serial = [np.load(os.path.join(str(tmp_path), "rank%d_0.npz" % r)) for r in range(world)]
+    over = [np.load(os.path.join(str(tmp_path), "rank%d_1.npz" % r)) for r in range(world)]
+    assert [(int(s["first"]), int(s["last"])) for s in serial] == [(0, 38), (38, 75)]       # uneven remainder
+    for r in range(world):
+        assert abs(serial[r]["loss"][0] - loss) <= 1e-12 * abs(loss)
+        assert over[r]["loss"][0] == serial[r]["loss"][0]
+        for i, ref in enumerate(dW + db):
+            assert np.allclose(serial[r]["arr_%d" % i], ref, rtol=1e-12, atol=1e-14)
+            # launched group by group or in one go: the same additions, the same bits
+            assert np.array_equal(over[r]["arr_%d" % i], serial[r]["arr_%d" % i])
+            if ordered:
+                assert np.array_equal(over[0]["arr_%d" % i], over[1]["arr_%d" % i])
