@@ -50,7 +50,17 @@ NOMINAL_TF32_OVER_BF16 = 0.5        # dense TF32 tensor rate is half the BF16 ra
 # dominant kernel, captured on a smaller batch and scaled by the pattern count, to which these products' traffic is
 # proportional.  Reported only while the library still is the version the counters were taken on; null otherwise.
 NCU_TRAFFIC = {
-    "library_version": -1,
+    "library_version": 109,
+    # captured at 16384 patterns (x4); in 16-bit mode at 32768 patterns (x2)
+    ("config3", "3xtf32", (3203, 481, 65536)): 4 * (302.14912e6 + 22.673664e6),
+    ("config3", "3xtf32", (65536, 480, 3203)): 4 * (310.02726e6 + 23.085568e6),
+    ("config3", "3xtf32", (65536, 3203, 480)): 4 * (77.086720e6 + 166.95372e6),
+    ("config3", "tf32", (65536, 3203, 480)): 4 * (39.002112e6 + 162.37900e6),
+    ("config3", "tf32", (65536, 480, 3203)): 4 * (256.99609e6 + 22.658560e6),
+    ("config3", "tf32", (3203, 481, 65536)): 4 * (250.86515e6 + 21.920000e6),
+    ("config3", "bf16", (65536, 3203, 480)): 2 * (38.322688e6 + 174.92428e6),
+    ("config3", "bf16", (65536, 480, 3203)): 2 * (251.78496e6 + 21.462784e6),
+    ("config3", "bf16", (3203, 481, 65536)): 2 * (253.33120e6 + 21.330432e6),
 }
 # cuBLAS through torch.matmul, 8192^3, on this machine's B200s (`--workload peaks`): TF32 allowed, best of 10 isolated
 # calls and 4 s back to back under the power cap (SM clock 1042 MHz of 1965).  Printed beside the peak the fractions use.
