@@ -446,15 +446,24 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                 tma_store_3d(&map_c, smem_u32(blk), c0, r0w, EPI == EPI_PARTIAL ? sp : 0);
                                 bulk_commit();
                             }
-                        } else if (rv) {
-                            float* dst = base + r * ld + c0;
-                            if ((EPI == EPI_PARTIAL || c_vec) && full) {
+                        } else {
+                            // rows TMA cannot address (a leading dimension that is not a multiple of four, a base that is not
+                            // 16-byte aligned): through the same staging block, then row by row in 128-byte runs by the warp
+                            uint8_t* blk = next_block();
+                            float4* rowp = reinterpret_cast<float4*>(blk + lane * 128);
 #pragma unroll
-                                for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
+                            for (int j = 0; j < 8; ++j)
+                                rowp[j ^ (lane & 7)] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            __syncwarp();
+                            const int rows_here = min(32, (int)(d.M - r0w));
+                            if (lane < nvalid) {
+                                float* dst = base + (int64_t)r0w * ld + c0 + lane;
+                                for (int rr = 0; rr < rows_here; ++rr) {
+                                    const float* src = reinterpret_cast<const float*>(blk + rr * 128 + ((((lane >> 2) ^ (rr & 7)) << 4) | ((lane & 3) << 2)));
+                                    dst[(int64_t)rr * ld] = *src;
+                                }
                             }
+                            __syncwarp();
                         }
                     }
                 }
