@@ -58,9 +58,9 @@ NCU_TRAFFIC = {
     ("config3", "tf32", (65536, 3203, 480)): 4 * (39.002112e6 + 162.37900e6),
     ("config3", "tf32", (65536, 480, 3203)): 4 * (256.99609e6 + 22.658560e6),
     ("config3", "tf32", (3203, 481, 65536)): 4 * (250.86515e6 + 21.920000e6),
-    ("config3", "bf16", (65536, 3203, 480)): 2 * (38.322688e6 + 174.92428e6),
-    ("config3", "bf16", (65536, 480, 3203)): 2 * (251.78496e6 + 21.462784e6),
-    ("config3", "bf16", (3203, 481, 65536)): 2 * (253.33120e6 + 21.330432e6),
+    ("config3", "bf16", (65536, 3203, 480)): 2 * (38.447872e6 + 175.91628e6),
+    ("config3", "bf16", (65536, 480, 3203)): 2 * (249.72902e6 + 20.953344e6),
+    ("config3", "bf16", (3203, 481, 65536)): 2 * (253.34092e6 + 21.497088e6),
 }
 # cuBLAS through torch.matmul, 8192^3, on this machine's B200s (`--workload peaks`): TF32 allowed, best of 10 isolated
 # calls and 4 s back to back under the power cap (SM clock 1042 MHz of 1965).  Printed beside the peak the fractions use.
